@@ -1,0 +1,153 @@
+/*
+ * chicle.h -- C ABI of libchicle: one CoCoA round for generalised linear models on one NVIDIA B200.
+ *
+ * A round (paper Sec. 2.1, Eq. 1 and Eq. 2; Sec. 2.2 "CoCoA"; Sec. 5.1 "CoCoA"): K uni-task partitions of the
+ * coordinates each run a sequential stochastic coordinate-descent solver against a private copy of the shared
+ * vector v, the K updates are added into v, and the duality gap (the paper's convergence metric, Sec. 4.1 and
+ * Sec. 5) can be evaluated. Every step runs in CUDA kernels of this library; there is no host fallback.
+ *
+ * Problem:   P(w) = (1/n) sum_i loss_i(x_i . w) + (lambda/2) |w|^2
+ *   - hinge and logistic: solved in the dual. Coordinates are the n examples (rows of X, CSR or dense
+ *     row-major), state alpha in R^n (signed: alpha_i = y_i a_i, a_i in [0,1]), shared vector
+ *     v = X^T alpha in R^d, w = v / (lambda n).
+ *   - ridge, loss_i(z) = (z - y_i)^2 / 2: solved in the primal over feature partitions. Coordinates are the d
+ *     columns of X (CSC), state w in R^d, shared vector v = X w in R^n.
+ *
+ * Conventions
+ *   - Every call returns a chicle_status_t. No C++ exception crosses this boundary. Out-parameters are left
+ *     untouched on error. After any error other than CHICLE_ERR_CUDA the handle is unchanged and usable.
+ *   - All pointers named host_* are host memory; chicle_matrix_t says where its arrays live. The library copies
+ *     what it needs at create time: the caller keeps ownership of everything it passes and may free it as soon
+ *     as the call returns. Everything the library allocates is released by chicle_glm_destroy.
+ *   - One handle is bound to one device and one stream, and is not thread-safe. Calls enqueue work on that
+ *     stream; calls that return host scalars or copy to host memory synchronise the stream.
+ *   - Kernels never trap. A device-side problem (a bounded wait that ran out, a non-finite step) is recorded in a
+ *     status word that the next synchronising call returns as CHICLE_ERR_TIMEOUT / CHICLE_ERR_NUMERIC.
+ *   - State machine (paper Sec. 3, ownership contract: data moves only between iterations):
+ *       create -> partition -> { cocoa_round | duality_gap | partition | get_* | set_state }*
+ *     chicle_cocoa_round before the first chicle_partition returns CHICLE_ERR_BAD_STATE. chicle_partition keeps
+ *     alpha, v and the round counter (per-sample state travels with its sample, Sec. 4.4).
+ */
+#ifndef CHICLE_H
+#define CHICLE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct chicle_glm chicle_glm_t; /* opaque, owned by the library */
+
+typedef enum {
+    CHICLE_OK = 0,
+    CHICLE_ERR_INVALID_ARG = 1,
+    CHICLE_ERR_BAD_STATE = 2,
+    CHICLE_ERR_OOM = 3,
+    CHICLE_ERR_CUDA = 4,
+    CHICLE_ERR_UNSUPPORTED = 5,
+    CHICLE_ERR_NUMERIC = 6,
+    CHICLE_ERR_TIMEOUT = 7
+} chicle_status_t;
+
+typedef enum { CHICLE_LOSS_HINGE_DUAL = 0, CHICLE_LOSS_LOGISTIC_DUAL = 1, CHICLE_LOSS_RIDGE_PRIMAL = 2 } chicle_loss_t;
+typedef enum { CHICLE_FMT_DENSE_ROWMAJOR = 0, CHICLE_FMT_CSR = 1, CHICLE_FMT_CSC = 2 } chicle_format_t;
+typedef enum { CHICLE_MEM_HOST = 0, CHICLE_MEM_DEVICE = 1 } chicle_memspace_t;
+
+/* Caller-owned description of X (n_rows examples by n_cols features). All arrays live in `space`.
+ *   dense:  values[i*ld + j], ld >= n_cols, indptr = indices = NULL, nnz ignored.
+ *   CSR:    indptr[n_rows+1], indices[nnz] column ids, values[nnz]; ids unique inside a row.
+ *   CSC:    indptr[n_cols+1], indices[nnz] row ids,    values[nnz]; ids unique inside a column.
+ * Hinge and logistic accept dense or CSR; ridge accepts CSC. Any other pairing is CHICLE_ERR_UNSUPPORTED. */
+typedef struct {
+    chicle_format_t fmt;
+    chicle_memspace_t space;
+    int64_t n_rows, n_cols, nnz, ld;
+    const int64_t *indptr;
+    const int32_t *indices;
+    const float *values;
+} chicle_matrix_t;
+
+/* Optional device allocator (for example one backed by a framework's caching allocator). Both callbacks or
+ * neither; NULL struct or NULL callbacks select cudaMalloc / cudaFree on the handle's device. `alloc` returns
+ * NULL on failure; returned pointers must be 256-byte aligned device memory. */
+typedef struct {
+    void *(*alloc)(void *ctx, size_t bytes);
+    void (*free)(void *ctx, void *ptr);
+    void *ctx;
+} chicle_allocator_t;
+
+/* Device timings of one round in milliseconds (CUDA events on the handle's stream). */
+typedef struct {
+    float ms_permutation; /* a2: visiting orders of this round                                  */
+    float ms_local;       /* a3+a4: local SCD solvers                                           */
+    float ms_reduce;      /* a5: v += sum_k dv_k                                                */
+    float ms_total;       /* whole round                                                        */
+    int64_t steps;        /* coordinate steps taken in this round, all partitions               */
+    int32_t solver_variant; /* 0 dense/shared-memory, 1 sparse/shared-memory, 2 sparse/global  */
+    int32_t reserved;
+} chicle_round_stats_t;
+
+/* Create a training problem (Sec. 2.2, Sec. 5.1: a GLM trained by CoCoA with a local SCD solver; Sec. 4.4:
+ * samples and their per-sample state are held together). Copies X and the labels to `device`, computes the
+ * squared norms of the coordinate vectors, zeroes alpha (or w) and v. `labels` has n_rows entries in X->space:
+ * +1/-1 for hinge and logistic (anything else: CHICLE_ERR_INVALID_ARG), real targets for ridge. NaN or Inf in
+ * values or labels: CHICLE_ERR_NUMERIC. `cuda_stream` is a cudaStream_t (NULL = the legacy default stream).
+ * Synchronises the stream before returning. On success *out receives the handle. */
+chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels, float lambda, chicle_loss_t loss,
+                                  int device, void *cuda_stream, const chicle_allocator_t *alloc,
+                                  chicle_glm_t **out);
+
+/* Random equal split of the coordinates into K disjoint covering partitions (Sec. 2.1: disjoint partitions D_k;
+ * Sec. 3: the data parallelism can change between iterations; Sec. 6: data is assigned to tasks at random).
+ * Integer rule: ids are ordered by mix64(mix64(seed) ^ id) (mix64 = one SplitMix64 output for that state) and
+ * cut into K consecutive blocks, the first n mod K one longer. 1 <= K <= number of coordinates. Legal only
+ * between rounds; keeps alpha, v and the round counter; (re)allocates the per-partition workspaces. */
+chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed);
+
+/* One CoCoA round (Sec. 2.1 Eq. 1, Eq. 2 and worker structure with L = 1; Sec. 5.1: SCD local solver, sigma =
+ * number of tasks). Each partition draws this round's seeded visiting order (members ordered by
+ * mix64(mix64(seed ^ 0xD1B54A32D192ED03) ^ mix64(round * 2^32 + epoch) ^ id)), walks it strictly in order for H
+ * coordinate steps (H = 0: one local epoch, i.e. as many steps as the partition has coordinates) against
+ * v_local = v + sigma' * (its own update so far), then v += sum_k dv_k in ascending k and the round counter
+ * advances. sigma_prime > 0; sigma' >= K guarantees dual ascent. Asynchronous unless `stats` is non-NULL, in
+ * which case the stream is synchronised and *stats filled. */
+chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime, chicle_round_stats_t *stats);
+
+/* Duality gap P(w(alpha)) - D(alpha) of the current state (Sec. 4.1, Sec. 5: the metric solvers report), with
+ * fp64 accumulation in a fixed order. host_gap / host_primal / host_dual may each be NULL. Synchronises. */
+chicle_status_t chicle_duality_gap(chicle_glm_t *h, double *host_gap, double *host_primal, double *host_dual);
+
+/* Copy out the state. `len` must equal the array's length: alpha has one entry per coordinate (n_rows for the
+ * dual losses, n_cols = w for ridge); v has n_cols entries for the dual losses and n_rows for ridge. `space` says
+ * where `out` lives. Synchronises. */
+chicle_status_t chicle_get_alpha(chicle_glm_t *h, float *out, int64_t len, chicle_memspace_t space);
+chicle_status_t chicle_get_v(chicle_glm_t *h, float *out, int64_t len, chicle_memspace_t space);
+
+/* Partition map: host_owner[c] = partition of coordinate c; len = number of coordinates. Synchronises. */
+chicle_status_t chicle_get_partition(chicle_glm_t *h, int32_t *host_owner, int64_t len);
+
+/* Visiting order of partition k in local epoch 0 of round `round` under the current partition (any round >= 0, not
+ * only the current one). len must equal the partition's size. Synchronises. */
+chicle_status_t chicle_get_permutation(chicle_glm_t *h, int64_t round, int32_t k, int32_t *host_out, int64_t len);
+
+/* Overwrite the state (checkpoint restore, or re-synchronising with an external trajectory). host_alpha has one
+ * entry per coordinate; host_v may be NULL, in which case v is recomputed from alpha on the device
+ * (v = X^T alpha, or X w). `round` >= 0 becomes the round counter. Synchronises. */
+chicle_status_t chicle_set_state(chicle_glm_t *h, const float *host_alpha, const float *host_v, int64_t round);
+
+/* Current round counter, partition count and coordinate / shared-vector lengths; any pointer may be NULL. */
+chicle_status_t chicle_get_info(const chicle_glm_t *h, int64_t *round, int32_t *K, int64_t *n_coord, int64_t *dim);
+
+/* Text of the last error on this handle (library-owned, valid until the next call on the handle). With h = NULL:
+ * the text of the last failed chicle_glm_create on this thread. Never NULL. */
+const char *chicle_last_error(const chicle_glm_t *h);
+
+/* Release everything the handle owns. NULL is allowed. */
+void chicle_glm_destroy(chicle_glm_t *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CHICLE_H */

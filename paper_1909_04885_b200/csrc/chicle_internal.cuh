@@ -1,0 +1,116 @@
+// Internal declarations shared by the translation units of libchicle (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+
+#include "chicle.h"
+
+namespace chicle {
+
+// ---- device status word (bit set by kernels, read by synchronising host calls) -------------------------
+enum : uint32_t {
+    ST_NONFINITE_INPUT = 1u << 0,  // NaN/Inf in values or labels
+    ST_BAD_LABEL = 1u << 1,        // label not +-1 for a dual loss
+    ST_BAD_INDEX = 1u << 2,        // index outside [0, dim) or indptr not monotone
+    ST_WAIT_TIMEOUT = 1u << 3,     // a bounded wait inside a kernel ran out
+    ST_NONFINITE_STEP = 1u << 4,   // a coordinate step produced NaN/Inf
+};
+
+// One SplitMix64 output for state x (published generator; a bijection on 64-bit words).
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t x)
+{
+    uint64_t z = x + 0x9E3779B97F4A7C15ULL;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+constexpr uint64_t kPermStream = 0xD1B54A32D192ED03ULL;
+
+// ---- radix sort over (64-bit key, 32-bit value) pairs -------------------------------------------------------
+constexpr int kSortThreads = 256;
+constexpr int kSortItems = 16;
+constexpr int kSortTile = kSortThreads * kSortItems;  // elements per block and pass
+
+struct SortWorkspace {
+    uint64_t *keys[2] = {nullptr, nullptr};
+    int32_t *vals[2] = {nullptr, nullptr};
+    uint32_t *hist = nullptr;      // 256 * nblk digit-major counters
+    uint32_t *scan_sums = nullptr; // one per scan tile
+    int64_t capacity = 0;          // elements
+    int nblk = 0;
+};
+
+size_t sort_hist_entries(int64_t n);
+size_t sort_scan_tiles(int64_t n);
+
+// Stable LSD pass on 8 bits. digit = (keys_in[i] >> shift) & 255 when owner == nullptr, else
+// (owner[vals_in[i]] >> shift) & 255. keys may be nullptr in owner mode (only values move).
+cudaError_t radix_pass(const uint64_t *keys_in, const int32_t *vals_in, uint64_t *keys_out, int32_t *vals_out,
+                       const int32_t *owner, int64_t n, int shift, uint32_t *hist, uint32_t *scan_sums,
+                       cudaStream_t stream);
+
+// ---- handle -------------------------------------------------------------------------------------------------
+struct Glm {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    chicle_allocator_t alloc{nullptr, nullptr, nullptr};
+    chicle_loss_t loss = CHICLE_LOSS_HINGE_DUAL;
+    chicle_format_t fmt = CHICLE_FMT_DENSE_ROWMAJOR;
+    int64_t n_rows = 0, n_cols = 0, nnz = 0;
+    int64_t n_coord = 0; // coordinates: rows (dual losses) or columns (ridge)
+    int64_t dim = 0;     // length of the shared vector
+    int64_t n_examples = 0;
+    float lambda = 0.f;
+
+    // coordinate-major matrix on the device (dense: indptr/indices null, row c at values + c*dim)
+    int64_t *indptr = nullptr;
+    int32_t *indices = nullptr;
+    float *values = nullptr;
+    float *labels = nullptr; // per example
+    float *sqnorm = nullptr; // per coordinate
+    float *alpha = nullptr;  // per coordinate: signed dual variable, or w for ridge
+    float *v = nullptr;      // shared vector, dim
+    float *resid = nullptr;  // ridge only: v - y, refreshed by the reduction kernel
+
+    // partition
+    int32_t K = 0;
+    uint64_t seed = 0;
+    int32_t *owner = nullptr;   // n_coord
+    int32_t *members = nullptr; // n_coord, grouped by partition, ascending id inside
+    int64_t *part_off = nullptr; // K+1 (device)
+    int64_t *h_part_off = nullptr; // K+1 (host)
+    int32_t *perm = nullptr;    // epochs * n_coord
+    int64_t perm_epochs = 0;
+    float *U = nullptr;         // K * dim: per-partition accumulated update, zero between rounds
+    int64_t U_rows = 0;
+
+    SortWorkspace sortws;
+    double *gap_partials = nullptr; // gap kernel partial sums
+    int gap_blocks = 0;
+    double *gap_out = nullptr;      // 8 doubles on the device
+    uint32_t *d_status = nullptr;
+    uint32_t *h_status = nullptr;   // pinned
+    double *h_gap = nullptr;        // pinned, 8 doubles
+
+    int64_t round = 0;
+    int sm_count = 148;
+    int max_smem_optin = 0;
+    cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    std::string err;
+};
+
+// ---- kernels' host launchers (each returns the launch error, work is enqueued on g.stream) -----------------
+cudaError_t launch_validate(Glm &g);
+cudaError_t launch_sqnorm(Glm &g);
+cudaError_t launch_partition(Glm &g, int32_t K, uint64_t seed);           // fills owner, members
+cudaError_t launch_permutation(Glm &g, int64_t round, int64_t epochs);    // fills perm[epochs * n_coord]
+cudaError_t launch_local_solver(Glm &g, int64_t H, float sigma_prime, int *variant);
+cudaError_t launch_reduce(Glm &g);                                        // v += sum_k U_k ; U = 0 ; resid
+cudaError_t launch_gap(Glm &g);                                           // fills gap_out[0..2]
+cudaError_t launch_shared_vector(Glm &g);                                 // v = X^T alpha (or X w) from scratch
+cudaError_t launch_refresh_resid(Glm &g);                                 // ridge: resid = v - y
+
+} // namespace chicle

@@ -1,0 +1,530 @@
+// Local stochastic coordinate-descent solvers: one CTA per partition, walking the partition's visiting order
+// strictly in order (paper Sec. 2.1 worker structure with L = 1; Sec. 2.2 and Sec. 5.1: SCD local solver).
+//
+// Roles inside a CTA
+//   warp 0        the chain: per step one dot product (lanes over the coordinate's entries, butterfly
+//                 reduction), the scalar step in registers, the scatter into the local model.
+//   warps 1..P    producers: run ahead of the chain and stage everything a step needs that does not depend on
+//                 earlier steps into a ring of shared-memory slots -- the coordinate id from the visiting order,
+//                 its entries, the read-only part of the shared vector at those entries (v is constant during a
+//                 round), and per-coordinate constants with their divisions already done. Copies are cp.async;
+//                 a slot is handed over through an mbarrier that the copies themselves arrive on.
+//
+// Local model: v_local = v + sigma' * U_k, where U_k is the partition's own accumulated update.
+//   dense rows   v_local and U_k live in shared memory; U_k is written out once at the end.
+//   sparse       U_k lives in global memory (one row of the K x dim workspace, zero at round start) and is only
+//                ever touched by this CTA, so it stays in this SM's L1 / the L2; v is gathered by the producers.
+//
+// Every wait is bounded; when one runs out the kernel records it in the status word and all roles return.
+#include <math_constants.h>
+
+#include "chicle_internal.cuh"
+
+namespace chicle {
+
+namespace {
+
+constexpr int kProdWarps = 4;
+constexpr int kGroup = 4;              // packets a producer keeps in flight
+constexpr int kSparseCap = 128;        // entries a sparse slot can hold; longer coordinates take the slow path
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kNewtonIters = 5;
+
+struct SlotHdr {
+    int64_t row_start;
+    int32_t coord;
+    int32_t nnz;
+    float p0, p1, p2, p3;
+    int32_t pad[2];
+};
+static_assert(sizeof(SlotHdr) == 40 || sizeof(SlotHdr) == 48, "header size");
+
+struct SolverParams {
+    const int64_t *indptr;
+    const int32_t *indices;
+    const float *values;
+    const float *labels;
+    const float *sqnorm;
+    float *alpha;
+    const float *vbase; // v (dual losses) or v - y (ridge)
+    float *U;           // K x dim
+    const int64_t *part_off;
+    const int32_t *perm; // epochs x n_coord
+    uint32_t *status;
+    int64_t n_coord, dim, H;
+    float lam_n, inv_n, lambda, sigma;
+    int cap, nslot, multi_epoch;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t a, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(a), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t a)
+{
+    asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"(a) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t a, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(a), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Bounded wait. Returns false when the CTA is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status)
+{
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 31u) == 31u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicOr(status, ST_WAIT_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// Scalar steps. `dot` is x_c . v_local (dual) or c_j . (v_local - y) (ridge). Returns delta and the new state.
+template <int LOSS>
+__device__ __forceinline__ void coordinate_step(float dot, const SlotHdr &h, float &delta, float &new_state)
+{
+    if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+        // p0 = 1/n, p1 = w_j, p2 = 1 / (sigma' |c_j|^2 / n + lambda), p3 = lambda
+        const float g = fmaf(dot, h.p0, h.p3 * h.p1);
+        delta = -g * h.p2;
+        new_state = h.p1 + delta;
+    } else if (LOSS == CHICLE_LOSS_HINGE_DUAL) {
+        // p0 = y / (lambda n), p1 = a, p2 = lambda n / (sigma' |x|^2) (inf for a zero row), p3 = y
+        const float m = dot * h.p0;
+        const float t = fmaf(1.0f - m, h.p2, h.p1);
+        const float a_new = fminf(fmaxf(t, 0.0f), 1.0f);
+        delta = h.p3 * (a_new - h.p1);
+        new_state = h.p3 * a_new;
+    } else {
+        // logistic: p0 = y / (lambda n), p1 = a, p2 = q = sigma' |x|^2 / (lambda n), p3 = y.
+        // Root of z + q sigmoid(z) = c on its convex branch (after reflecting a positive root), Newton from a
+        // Lambert-W-like start, fixed iteration count.
+        const float q = h.p2, a = h.p1;
+        const float m = dot * h.p0;
+        float c = fmaf(q, a, -m);
+        const bool flip = c > 0.5f * q;
+        if (flip) c = q - c;
+        const float kappa = q > 0.0f ? __logf(q) + c : -CUDART_INF_F;
+        float z = kappa <= 0.0f ? fminf(c, 0.0f) : fminf(c - (kappa - __logf(1.0f + kappa)), 0.0f);
+#pragma unroll
+        for (int it = 0; it < kNewtonIters; ++it) {
+            const float e = __expf(z);
+            const float r = __frcp_rn(1.0f + e);
+            const float p = e * r;
+            const float F = fmaf(q, p, z) - c;
+            const float Fp = fmaf(q * p, r, 1.0f); // 1 + q p (1 - p), 1 - p = 1 / (1 + e)
+            z = fminf(z - __fdividef(F, Fp), 0.0f);
+        }
+        const float e = __expf(z);
+        const float r = __frcp_rn(1.0f + e);
+        const float a_new = flip ? r : e * r;
+        delta = h.p3 * (a_new - a);
+        new_state = h.p3 * a_new;
+    }
+}
+
+template <int LOSS, bool DENSE>
+__global__ void __launch_bounds__(32 * (1 + kProdWarps), 1) k_local_scd(const SolverParams P)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int k = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nslot = P.nslot, cap = P.cap;
+
+    // ---- carve shared memory
+    uint64_t *bar_full = reinterpret_cast<uint64_t *>(smem_raw);
+    uint64_t *bar_empty = bar_full + nslot;
+    volatile long long *progress = reinterpret_cast<volatile long long *>(bar_empty + nslot);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(progress + 1);
+    SlotHdr *hdrs = reinterpret_cast<SlotHdr *>(smem_raw + ((2 * nslot + 2) * 8 + 15) / 16 * 16);
+    float *fbase = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(hdrs) +
+                                             ((size_t)nslot * sizeof(SlotHdr) + 127) / 128 * 128);
+    float *vloc = nullptr, *dv = nullptr, *s_val, *s_base = nullptr;
+    int32_t *s_idx = nullptr;
+    if (DENSE) {
+        vloc = fbase;
+        dv = fbase + cap;
+        s_val = fbase + 2 * cap;
+    } else {
+        s_val = fbase;
+        s_base = fbase + (size_t)nslot * cap;
+        s_idx = reinterpret_cast<int32_t *>(fbase + 2 * (size_t)nslot * cap);
+    }
+
+    const int64_t off = P.part_off[k];
+    const int64_t nk = P.part_off[k + 1] - off;
+    const int64_t steps = nk <= 0 ? 0 : (P.H == 0 ? nk : P.H);
+
+    if (threadIdx.x == 0) {
+        *progress = 0;
+        *abort_flag = 0;
+    }
+    for (int s = threadIdx.x; s < nslot; s += blockDim.x) {
+        mbar_init(smem_u32(&bar_full[s]), 33);  // 32 copy-completion arrivals + 1 plain arrival
+        mbar_init(smem_u32(&bar_empty[s]), 32); // the chain warp's lanes
+    }
+    if (DENSE) {
+        for (int j = threadIdx.x; j < cap; j += blockDim.x) {
+            vloc[j] = j < P.dim ? P.vbase[j] : 0.0f;
+            dv[j] = 0.0f;
+        }
+    }
+    __syncthreads();
+    if (steps == 0) {
+        if (DENSE)
+            for (int j = threadIdx.x; j < P.dim; j += blockDim.x) P.U[(size_t)k * P.dim + j] = 0.0f;
+        return;
+    }
+    float *Uk = P.U + (size_t)k * (size_t)P.dim;
+
+    if (warp == 0) {
+        // =============================== the chain ===============================
+        for (int64_t t = 0; t < steps; ++t) {
+            const int s = (int)(t % nslot);
+            const uint32_t use = (uint32_t)(t / nslot);
+            if (!mbar_wait(smem_u32(&bar_full[s]), use & 1u, abort_flag, P.status)) return;
+            const SlotHdr h = hdrs[s];
+            float acc = 0.0f;
+            float delta, new_state;
+            if (DENSE) {
+                const float *row = s_val + (size_t)s * cap;
+                for (int j = lane; j < (int)P.dim; j += 32) acc = fmaf(row[j], vloc[j], acc);
+                acc = warp_sum(acc);
+                coordinate_step<LOSS>(acc, h, delta, new_state);
+                if (!(fabsf(delta) <= CUDART_MAX_NORMAL_F)) {
+                    if (lane == 0) atomicOr(P.status, ST_NONFINITE_STEP);
+                    delta = 0.0f;
+                    new_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? h.p1 : h.p3 * h.p1;
+                }
+                if (delta != 0.0f) {
+                    const float sd = P.sigma * delta;
+                    for (int j = lane; j < (int)P.dim; j += 32) {
+                        const float x = row[j];
+                        vloc[j] = fmaf(sd, x, vloc[j]);
+                        dv[j] = fmaf(delta, x, dv[j]);
+                    }
+                }
+            } else if (h.nnz <= cap) {
+                const int32_t *ix = s_idx + (size_t)s * cap;
+                const float *xv = s_val + (size_t)s * cap;
+                const float *bv = s_base + (size_t)s * cap;
+                // first two strided entries stay in registers (covers up to 64 entries without re-reading)
+                int32_t j0 = 0, j1 = 0;
+                float x0 = 0.0f, x1 = 0.0f, u0 = 0.0f, u1 = 0.0f;
+                if (lane < h.nnz) {
+                    j0 = ix[lane];
+                    x0 = xv[lane];
+                    u0 = Uk[j0];
+                    acc = x0 * fmaf(P.sigma, u0, bv[lane]);
+                }
+                if (lane + 32 < h.nnz) {
+                    j1 = ix[lane + 32];
+                    x1 = xv[lane + 32];
+                    u1 = Uk[j1];
+                    acc = fmaf(x1, fmaf(P.sigma, u1, bv[lane + 32]), acc);
+                }
+                for (int e = lane + 64; e < h.nnz; e += 32)
+                    acc = fmaf(xv[e], fmaf(P.sigma, Uk[ix[e]], bv[e]), acc);
+                acc = warp_sum(acc);
+                coordinate_step<LOSS>(acc, h, delta, new_state);
+                if (!(fabsf(delta) <= CUDART_MAX_NORMAL_F)) {
+                    if (lane == 0) atomicOr(P.status, ST_NONFINITE_STEP);
+                    delta = 0.0f;
+                    new_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? h.p1 : h.p3 * h.p1;
+                }
+                if (delta != 0.0f) {
+                    if (lane < h.nnz) Uk[j0] = fmaf(delta, x0, u0);
+                    if (lane + 32 < h.nnz) Uk[j1] = fmaf(delta, x1, u1);
+                    for (int e = lane + 64; e < h.nnz; e += 32) {
+                        const int32_t j = ix[e];
+                        Uk[j] = fmaf(delta, xv[e], Uk[j]);
+                    }
+                }
+            } else {
+                // slow path: a coordinate with more entries than a slot holds is read straight from global memory
+                const int32_t *ix = P.indices + h.row_start;
+                const float *xv = P.values + h.row_start;
+                for (int e = lane; e < h.nnz; e += 32) {
+                    const int32_t j = ix[e];
+                    acc = fmaf(xv[e], fmaf(P.sigma, Uk[j], P.vbase[j]), acc);
+                }
+                acc = warp_sum(acc);
+                coordinate_step<LOSS>(acc, h, delta, new_state);
+                if (!(fabsf(delta) <= CUDART_MAX_NORMAL_F)) {
+                    if (lane == 0) atomicOr(P.status, ST_NONFINITE_STEP);
+                    delta = 0.0f;
+                    new_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? h.p1 : h.p3 * h.p1;
+                }
+                if (delta != 0.0f)
+                    for (int e = lane; e < h.nnz; e += 32) {
+                        const int32_t j = ix[e];
+                        Uk[j] = fmaf(delta, xv[e], Uk[j]);
+                    }
+            }
+            if (lane == 0) P.alpha[h.coord] = new_state;
+            __syncwarp();
+            if (P.multi_epoch) {
+                __threadfence_block();
+                if (lane == 0) *progress = t + 1;
+            }
+            mbar_arrive(smem_u32(&bar_empty[s]));
+        }
+        if (DENSE) {
+            __syncwarp();
+            for (int j = lane; j < (int)P.dim; j += 32) Uk[j] = dv[j];
+        }
+    } else {
+        // =============================== producers ===============================
+        // Producer warp w owns the slots [w*batch, (w+1)*batch): batch b of `batch` consecutive steps goes to warp
+        // b mod P, so successive uses of a slot are always filled by the same warp and the parity waits on its
+        // "empty" barrier can never be more than one phase behind.
+        const int pw = warp - 1;
+        const int batch = nslot / kProdWarps;
+        const int64_t n_batches = (steps + batch - 1) / batch;
+        for (int64_t b = pw; b < n_batches; b += kProdWarps) {
+            const int64_t t0 = b * batch;
+            const int cnt = (int)((steps - t0) < batch ? (steps - t0) : batch);
+            const int64_t ep_first = t0 / nk, ep_last = (t0 + cnt - 1) / nk;
+            int32_t c = 0, nnz = 0;
+            int64_t rs = 0;
+            float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
+            for (int64_t ep = ep_first; ep <= ep_last; ++ep) {
+                // lanes [l_lo, l_hi) of this batch are steps of local epoch ep
+                const int l_lo = (int)(ep * nk > t0 ? ep * nk - t0 : 0);
+                const int l_hi = (int)((ep + 1) * nk - t0 < cnt ? (ep + 1) * nk - t0 : cnt);
+                if (ep > 0) {
+                    // alpha of a coordinate visited again in a later local epoch must be read after the chain
+                    // wrote it: wait until the chain has finished the previous epoch
+                    uint32_t it = 0;
+                    while (*progress < ep * nk) {
+                        if (*abort_flag) { cp_async_wait_all(); return; }
+                        if (++it > kSpinLimit) {
+                            *abort_flag = 1;
+                            atomicOr(P.status, ST_WAIT_TIMEOUT);
+                            cp_async_wait_all();
+                            return;
+                        }
+                        __nanosleep(64);
+                    }
+                    __threadfence_block();
+                }
+                // ---- per-step headers: lane l prepares step t0 + l
+                if (lane >= l_lo && lane < l_hi) {
+                    const int64_t pos = t0 + lane - ep * nk;
+                    c = P.perm[(size_t)ep * (size_t)P.n_coord + (size_t)(off + pos)];
+                    if (DENSE) {
+                        rs = (int64_t)c * P.dim;
+                        nnz = (int32_t)P.dim;
+                    } else {
+                        rs = P.indptr[c];
+                        nnz = (int32_t)(P.indptr[c + 1] - rs);
+                    }
+                    const float s = P.sqnorm[c];
+                    const float st = __ldcg(P.alpha + c);
+                    if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+                        p0 = P.inv_n;
+                        p1 = st;
+                        p2 = 1.0f / fmaf(P.sigma * s, P.inv_n, P.lambda);
+                        p3 = P.lambda;
+                    } else {
+                        const float y = P.labels[c];
+                        p0 = y / P.lam_n;
+                        p1 = y * st;
+                        p3 = y;
+                        if (LOSS == CHICLE_LOSS_HINGE_DUAL) p2 = s > 0.0f ? P.lam_n / (P.sigma * s) : CUDART_INF_F;
+                        else p2 = P.sigma * s / P.lam_n;
+                    }
+                }
+                // ---- stage the packets, kGroup at a time
+                for (int g0 = l_lo; g0 < l_hi; g0 += kGroup) {
+                    int32_t idxr[kGroup][kSparseCap / 32];
+                    int32_t g_nnz[kGroup];
+                    int64_t g_rs[kGroup];
+#pragma unroll
+                    for (int g = 0; g < kGroup; ++g) {
+                        const int l = g0 + g;
+                        g_nnz[g] = __shfl_sync(0xffffffffu, nnz, l & 31);
+                        g_rs[g] = __shfl_sync(0xffffffffu, rs, l & 31);
+                        if (l >= l_hi) g_nnz[g] = -1;
+                    }
+                    // wait for the slots, then issue the index loads of the whole group
+#pragma unroll
+                    for (int g = 0; g < kGroup; ++g) {
+                        if (g_nnz[g] < 0) continue;
+                        const int64_t t = t0 + g0 + g;
+                        const int s = (int)(t % nslot);
+                        const uint32_t use = (uint32_t)(t / nslot);
+                        if (use > 0 && !mbar_wait(smem_u32(&bar_empty[s]), (use - 1u) & 1u, abort_flag, P.status)) {
+                            cp_async_wait_all();
+                            return;
+                        }
+                        if (!DENSE && g_nnz[g] <= cap) {
+#pragma unroll
+                            for (int r = 0; r < kSparseCap / 32; ++r) {
+                                const int e = r * 32 + lane;
+                                idxr[g][r] = e < g_nnz[g] ? P.indices[g_rs[g] + e] : 0;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int g = 0; g < kGroup; ++g) {
+                        if (g_nnz[g] < 0) continue;
+                        const int l = g0 + g;
+                        const int64_t t = t0 + l;
+                        const int s = (int)(t % nslot);
+                        const uint32_t bar = smem_u32(&bar_full[s]);
+                        if (DENSE) {
+                            const float *src = P.values + g_rs[g];
+                            const uint32_t dst = smem_u32(s_val + (size_t)s * cap);
+                            if ((P.dim & 3) == 0) {
+                                for (int j4 = lane; j4 < (int)(P.dim >> 2); j4 += 32)
+                                    cp_async16(dst + 16u * j4, src + 4 * j4);
+                            } else {
+                                for (int j = lane; j < (int)P.dim; j += 32) cp_async4(dst + 4u * j, src + j);
+                            }
+                        } else if (g_nnz[g] <= cap) {
+                            const uint32_t dval = smem_u32(s_val + (size_t)s * cap);
+                            const uint32_t dbase = smem_u32(s_base + (size_t)s * cap);
+                            int32_t *dix = s_idx + (size_t)s * cap;
+#pragma unroll
+                            for (int r = 0; r < kSparseCap / 32; ++r) {
+                                const int e = r * 32 + lane;
+                                if (e < g_nnz[g]) {
+                                    cp_async4(dval + 4u * e, P.values + g_rs[g] + e);
+                                    cp_async4(dbase + 4u * e, P.vbase + idxr[g][r]);
+                                    dix[e] = idxr[g][r];
+                                }
+                            }
+                        }
+                        cp_async_arrive_noinc(bar);
+                        // header: every lane holds its own step's constants; lane l writes the header of step l
+                        if (lane == l) {
+                            SlotHdr hd;
+                            hd.row_start = rs;
+                            hd.coord = c;
+                            hd.nnz = nnz;
+                            hd.p0 = p0; hd.p1 = p1; hd.p2 = p2; hd.p3 = p3;
+                            hd.pad[0] = hd.pad[1] = 0;
+                            hdrs[s] = hd;
+                        }
+                        __syncwarp();
+                        if (lane == l) mbar_arrive(bar);
+                    }
+                }
+            }
+        }
+        cp_async_wait_all();
+    }
+}
+
+template <int LOSS, bool DENSE>
+cudaError_t launch_variant(Glm &g, const SolverParams &P, size_t smem)
+{
+    auto kern = k_local_scd<LOSS, DENSE>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<g.K, 32 * (1 + kProdWarps), smem, g.stream>>>(P);
+    return cudaGetLastError();
+}
+
+size_t smem_bytes(bool dense, int cap, int nslot)
+{
+    size_t s = ((size_t)(2 * nslot + 2) * 8 + 15) / 16 * 16;
+    s += ((size_t)nslot * sizeof(SlotHdr) + 127) / 128 * 128;
+    if (dense) s += (size_t)(2 + nslot) * cap * 4;
+    else s += (size_t)3 * nslot * cap * 4;
+    return s + 128;
+}
+
+} // namespace
+
+bool solver_supports_dense(int64_t dim, int max_smem_optin)
+{
+    if (dim > (1 << 20)) return false;
+    const int cap = (int)((dim + 31) / 32 * 32);
+    return smem_bytes(true, cap, 4) <= (size_t)max_smem_optin;
+}
+
+cudaError_t launch_local_solver(Glm &g, int64_t H, float sigma_prime, int *variant)
+{
+    SolverParams P{};
+    P.indptr = g.indptr;
+    P.indices = g.indices;
+    P.values = g.values;
+    P.labels = g.labels;
+    P.sqnorm = g.sqnorm;
+    P.alpha = g.alpha;
+    P.vbase = g.loss == CHICLE_LOSS_RIDGE_PRIMAL ? g.resid : g.v;
+    P.U = g.U;
+    P.part_off = g.part_off;
+    P.perm = g.perm;
+    P.status = g.d_status;
+    P.n_coord = g.n_coord;
+    P.dim = g.dim;
+    P.H = H;
+    P.lam_n = g.lambda * (float)g.n_examples;
+    P.inv_n = 1.0f / (float)g.n_examples;
+    P.lambda = g.lambda;
+    P.sigma = sigma_prime;
+    const int64_t min_nk = g.n_coord / g.K;
+    P.multi_epoch = (H != 0 && H > min_nk) ? 1 : 0;
+
+    const bool dense = g.fmt == CHICLE_FMT_DENSE_ROWMAJOR;
+    const size_t budget = (size_t)g.max_smem_optin;
+    int cap, nslot = 64; // a multiple of the producer warp count; each producer owns nslot / P slots
+    if (dense) {
+        cap = (int)((g.dim + 31) / 32 * 32);
+        while (nslot > 4 && smem_bytes(true, cap, nslot) > budget) nslot /= 2;
+        if (smem_bytes(true, cap, nslot) > budget) return cudaErrorInvalidConfiguration;
+        *variant = 0;
+    } else {
+        cap = kSparseCap;
+        while (nslot > 4 && smem_bytes(false, cap, nslot) > budget / 2) nslot /= 2; // leave room for L1
+        *variant = 2;
+    }
+    P.cap = cap;
+    P.nslot = nslot;
+    const size_t smem = smem_bytes(dense, cap, nslot);
+
+    switch (g.loss) {
+    case CHICLE_LOSS_HINGE_DUAL:
+        return dense ? launch_variant<CHICLE_LOSS_HINGE_DUAL, true>(g, P, smem)
+                     : launch_variant<CHICLE_LOSS_HINGE_DUAL, false>(g, P, smem);
+    case CHICLE_LOSS_LOGISTIC_DUAL:
+        return dense ? launch_variant<CHICLE_LOSS_LOGISTIC_DUAL, true>(g, P, smem)
+                     : launch_variant<CHICLE_LOSS_LOGISTIC_DUAL, false>(g, P, smem);
+    default:
+        return launch_variant<CHICLE_LOSS_RIDGE_PRIMAL, false>(g, P, smem);
+    }
+}
+
+} // namespace chicle

@@ -1,0 +1,350 @@
+// Streaming kernels: input validation, squared norms, aggregation of the K partition updates into the shared
+// vector (Eq. 2 with the updates added), the duality gap (the paper's convergence metric), and the from-scratch
+// shared vector used when a state is restored.
+#include <math_constants.h>
+
+#include "chicle_internal.cuh"
+
+namespace chicle {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarpsPerBlock = kThreads / 32;
+
+inline unsigned blocks_for(int64_t n, int t) { return (unsigned)((n + t - 1) / t); }
+
+__device__ __forceinline__ double warp_sum_d(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// ---------------------------------------------------------------------------------------- validation
+__global__ void k_validate_values(const float *__restrict__ x, int64_t n, uint32_t *status)
+{
+    bool bad = false;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        bad |= !(fabsf(x[i]) <= CUDART_MAX_NORMAL_F);
+    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicOr(status, ST_NONFINITE_INPUT);
+}
+
+__global__ void k_validate_labels(const float *__restrict__ y, int64_t n, int need_pm1, uint32_t *status)
+{
+    uint32_t bits = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const float t = y[i];
+        if (!(fabsf(t) <= CUDART_MAX_NORMAL_F)) bits |= ST_NONFINITE_INPUT;
+        else if (need_pm1 && t != 1.0f && t != -1.0f) bits |= ST_BAD_LABEL;
+    }
+    if (bits) atomicOr(status, bits);
+}
+
+__global__ void k_validate_structure(const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices,
+                                     int64_t n_coord, int64_t nnz, int64_t dim, uint32_t *status)
+{
+    bool bad = false;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t c = tid; c < n_coord; c += stride) bad |= indptr[c + 1] < indptr[c];
+    if (tid == 0) bad |= indptr[0] != 0 || indptr[n_coord] != nnz;
+    for (int64_t e = tid; e < nnz; e += stride) bad |= indices[e] < 0 || indices[e] >= dim;
+    if (bad) atomicOr(status, ST_BAD_INDEX);
+}
+
+// ---------------------------------------------------------------------------------------- squared norms
+__global__ void __launch_bounds__(kThreads)
+k_sqnorm(const int64_t *__restrict__ indptr, const float *__restrict__ values, int64_t n_coord, int64_t dim,
+         float *__restrict__ out)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t nw = (int64_t)gridDim.x * kWarpsPerBlock;
+    for (int64_t c = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); c < n_coord; c += nw) {
+        const int64_t b = indptr ? indptr[c] : c * dim;
+        const int64_t e = indptr ? indptr[c + 1] : b + dim;
+        double s = 0.0;
+        for (int64_t q = b + lane; q < e; q += 32) {
+            const double x = (double)values[q];
+            s = fma(x, x, s);
+        }
+        s = warp_sum_d(s);
+        if (lane == 0) out[c] = (float)s;
+    }
+}
+
+// ---------------------------------------------------------------------------------------- aggregation (a5)
+// v[j] += sum_k U[k][j] with k ascending and an fp64 accumulator; U is cleared for the next round; for ridge
+// the residual v - y that the next round's solvers gather from is refreshed in the same pass.
+template <int VEC>
+__global__ void __launch_bounds__(kThreads)
+k_reduce_updates(float *__restrict__ v, float *__restrict__ U, int K, int64_t dim, const float *__restrict__ y,
+                 float *__restrict__ resid)
+{
+    const int64_t nvec = dim / VEC;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (int64_t)gridDim.x * blockDim.x) {
+        double acc[VEC];
+        if (VEC == 4) {
+            const float4 t = reinterpret_cast<const float4 *>(v)[i];
+            acc[0] = t.x; acc[1 % VEC] = t.y; acc[2 % VEC] = t.z; acc[3 % VEC] = t.w;
+        } else {
+            acc[0] = v[i];
+        }
+#pragma unroll 8
+        for (int k = 0; k < K; ++k) {
+            if (VEC == 4) {
+                float4 *p = reinterpret_cast<float4 *>(U + (size_t)k * dim) + i;
+                const float4 t = *p;
+                acc[0] += t.x; acc[1 % VEC] += t.y; acc[2 % VEC] += t.z; acc[3 % VEC] += t.w;
+                *p = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else {
+                float *p = U + (size_t)k * dim + i;
+                acc[0] += *p;
+                *p = 0.f;
+            }
+        }
+        if (VEC == 4) {
+            const float4 o = make_float4((float)acc[0], (float)acc[1 % VEC], (float)acc[2 % VEC], (float)acc[3 % VEC]);
+            reinterpret_cast<float4 *>(v)[i] = o;
+            if (resid) {
+                const float4 t = reinterpret_cast<const float4 *>(y)[i];
+                reinterpret_cast<float4 *>(resid)[i] = make_float4(o.x - t.x, o.y - t.y, o.z - t.z, o.w - t.w);
+            }
+        } else {
+            const float o = (float)acc[0];
+            v[i] = o;
+            if (resid) resid[i] = o - y[i];
+        }
+    }
+}
+
+__global__ void k_resid(const float *__restrict__ v, const float *__restrict__ y, int64_t n, float *__restrict__ r)
+{
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        r[i] = v[i] - y[i];
+}
+
+// ---------------------------------------------------------------------------------------- duality gap (a6)
+// One pass over the coordinate-major matrix: a warp per coordinate computes its dot product with the shared
+// vector in fp64 and the coordinate's term; lane 0 of every warp keeps running fp64 sums over the coordinates it
+// was assigned (a fixed assignment), the block adds its warps in order and writes 4 partial sums; a second kernel
+// adds the blocks in order. Partials: dual losses {sum loss, sum gap term, |v|^2 slice, 0};
+// ridge {sum (c_j . r)^2, sum w_j^2, sum r^2 slice, sum r*y slice} with r = v - y.
+__device__ __forceinline__ double xlogx(double x) { return x > 0.0 ? x * log(x) : 0.0; }
+
+template <int LOSS>
+__global__ void __launch_bounds__(kThreads)
+k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices,
+               const float *__restrict__ values, const float *__restrict__ labels, const float *__restrict__ state,
+               const float *__restrict__ vec /* the shared vector */, const float *__restrict__ v,
+               int64_t n_coord, int64_t dim, double lam_n, double *__restrict__ partials)
+{
+    __shared__ double sh[kWarpsPerBlock][4];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t nw = (int64_t)gridDim.x * kWarpsPerBlock;
+    double s0 = 0.0, s1 = 0.0;
+    for (int64_t c = (int64_t)blockIdx.x * kWarpsPerBlock + warp; c < n_coord; c += nw) {
+        double dot = 0.0;
+        if (indptr) {
+            const int64_t b = indptr[c], e = indptr[c + 1];
+            if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+                for (int64_t q = b + lane; q < e; q += 32) {
+                    const int32_t r = indices[q];
+                    dot = fma((double)values[q], (double)vec[r] - (double)labels[r], dot);
+                }
+            } else {
+                for (int64_t q = b + lane; q < e; q += 32) dot = fma((double)values[q], (double)vec[indices[q]], dot);
+            }
+        } else {
+            const float *row = values + c * dim;
+            for (int64_t j = lane; j < dim; j += 32) dot = fma((double)row[j], (double)vec[j], dot);
+        }
+        dot = warp_sum_d(dot);
+        if (lane == 0) {
+            if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+                const double w = (double)state[c];
+                s0 += dot * dot;
+                s1 += w * w;
+            } else {
+                const double y = (double)labels[c];
+                const double mu = y * dot / lam_n;
+                double a = y * (double)state[c];
+                a = a < 0.0 ? 0.0 : (a > 1.0 ? 1.0 : a);
+                double l, conj;
+                if (LOSS == CHICLE_LOSS_HINGE_DUAL) {
+                    l = 1.0 - mu > 0.0 ? 1.0 - mu : 0.0;
+                    conj = -a;
+                } else {
+                    l = mu < 0.0 ? -mu + log1p(exp(mu)) : log1p(exp(-mu));
+                    conj = xlogx(a) + xlogx(1.0 - a);
+                }
+                s0 += l;
+                s1 += l + conj + a * mu;
+            }
+        }
+    }
+    // slice of the shared vector owned by this block
+    double s2 = 0.0, s3 = 0.0;
+    {
+        const int64_t chunk = (dim + gridDim.x - 1) / gridDim.x;
+        const int64_t b = (int64_t)blockIdx.x * chunk;
+        const int64_t e = b + chunk < dim ? b + chunk : dim;
+        for (int64_t j = b + threadIdx.x; j < e; j += kThreads) {
+            if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+                const double y = (double)labels[j]; // targets
+                const double r = (double)v[j] - y;
+                s2 = fma(r, r, s2);
+                s3 = fma(r, y, s3);
+            } else {
+                const double t = (double)v[j];
+                s2 = fma(t, t, s2);
+            }
+        }
+        s2 = warp_sum_d(s2);
+        s3 = warp_sum_d(s3);
+    }
+    if (lane == 0) {
+        sh[warp][0] = s0; sh[warp][1] = s1; sh[warp][2] = s2; sh[warp][3] = s3;
+    }
+    __syncthreads();
+    if (threadIdx.x < 4) {
+        double t = 0.0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) t += sh[w][threadIdx.x];
+        partials[(size_t)blockIdx.x * 4 + threadIdx.x] = t;
+    }
+}
+
+template <int LOSS>
+__global__ void k_gap_final(const double *__restrict__ partials, int nblocks, double n, double lambda,
+                            double *__restrict__ out)
+{
+    __shared__ double tot[4];
+    if (threadIdx.x < 4) {
+        double t = 0.0;
+        for (int b = 0; b < nblocks; ++b) t += partials[(size_t)b * 4 + threadIdx.x];
+        tot[threadIdx.x] = t;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double primal, dual;
+        if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+            const double cc = tot[0], ww = tot[1], rr = tot[2], ry = tot[3];
+            primal = rr / (2.0 * n) + 0.5 * lambda * ww;
+            dual = -(rr / (2.0 * n) + ry / n) - cc / (n * n * 2.0 * lambda);
+        } else {
+            const double lam_n = lambda * n;
+            primal = tot[0] / n + 0.5 * lambda * tot[2] / (lam_n * lam_n);
+            dual = primal - tot[1] / n;
+        }
+        out[0] = primal - dual;
+        out[1] = primal;
+        out[2] = dual;
+    }
+}
+
+// ---------------------------------------------------------------------------------------- v from scratch
+__global__ void __launch_bounds__(kThreads)
+k_shared_vector(const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices,
+                const float *__restrict__ values, const float *__restrict__ state, int64_t n_coord, int64_t dim,
+                float *__restrict__ v)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t nw = (int64_t)gridDim.x * kWarpsPerBlock;
+    for (int64_t c = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); c < n_coord; c += nw) {
+        const float s = state[c];
+        if (s == 0.0f) continue;
+        if (indptr) {
+            const int64_t b = indptr[c], e = indptr[c + 1];
+            for (int64_t q = b + lane; q < e; q += 32) atomicAdd(v + indices[q], s * values[q]);
+        } else {
+            const float *row = values + c * dim;
+            for (int64_t j = lane; j < dim; j += 32) atomicAdd(v + j, s * row[j]);
+        }
+    }
+}
+
+} // namespace
+
+cudaError_t launch_validate(Glm &g)
+{
+    const int64_t nvals = g.indptr ? g.nnz : g.n_coord * g.dim;
+    const unsigned grid = (unsigned)g.sm_count * 8;
+    k_validate_values<<<grid, kThreads, 0, g.stream>>>(g.values, nvals, g.d_status);
+    k_validate_labels<<<grid, kThreads, 0, g.stream>>>(g.labels, g.n_examples,
+                                                       g.loss != CHICLE_LOSS_RIDGE_PRIMAL, g.d_status);
+    if (g.indptr)
+        k_validate_structure<<<grid, kThreads, 0, g.stream>>>(g.indptr, g.indices, g.n_coord, g.nnz, g.dim,
+                                                              g.d_status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sqnorm(Glm &g)
+{
+    const unsigned grid = (unsigned)g.sm_count * 8;
+    k_sqnorm<<<grid, kThreads, 0, g.stream>>>(g.indptr, g.values, g.n_coord, g.dim, g.sqnorm);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reduce(Glm &g)
+{
+    const float *y = g.loss == CHICLE_LOSS_RIDGE_PRIMAL ? g.labels : nullptr;
+    float *resid = g.loss == CHICLE_LOSS_RIDGE_PRIMAL ? g.resid : nullptr;
+    if ((g.dim & 3) == 0) {
+        const int64_t nvec = g.dim / 4;
+        unsigned grid = blocks_for(nvec, kThreads);
+        if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
+        k_reduce_updates<4><<<grid, kThreads, 0, g.stream>>>(g.v, g.U, g.K, g.dim, y, resid);
+    } else {
+        unsigned grid = blocks_for(g.dim, kThreads);
+        if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
+        k_reduce_updates<1><<<grid, kThreads, 0, g.stream>>>(g.v, g.U, g.K, g.dim, y, resid);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_refresh_resid(Glm &g)
+{
+    if (g.loss != CHICLE_LOSS_RIDGE_PRIMAL) return cudaSuccess;
+    k_resid<<<(unsigned)g.sm_count * 4, kThreads, 0, g.stream>>>(g.v, g.labels, g.dim, g.resid);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gap(Glm &g)
+{
+    const int nb = g.gap_blocks;
+    const double n = (double)g.n_examples;
+    const double lam_n = (double)g.lambda * n;
+    switch (g.loss) {
+    case CHICLE_LOSS_HINGE_DUAL:
+        k_gap_partials<CHICLE_LOSS_HINGE_DUAL><<<nb, kThreads, 0, g.stream>>>(
+            g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord, g.dim, lam_n, g.gap_partials);
+        k_gap_final<CHICLE_LOSS_HINGE_DUAL><<<1, 32, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda, g.gap_out);
+        break;
+    case CHICLE_LOSS_LOGISTIC_DUAL:
+        k_gap_partials<CHICLE_LOSS_LOGISTIC_DUAL><<<nb, kThreads, 0, g.stream>>>(
+            g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord, g.dim, lam_n, g.gap_partials);
+        k_gap_final<CHICLE_LOSS_LOGISTIC_DUAL><<<1, 32, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda,
+                                                                        g.gap_out);
+        break;
+    default:
+        k_gap_partials<CHICLE_LOSS_RIDGE_PRIMAL><<<nb, kThreads, 0, g.stream>>>(
+            g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord, g.dim, lam_n, g.gap_partials);
+        k_gap_final<CHICLE_LOSS_RIDGE_PRIMAL><<<1, 32, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda,
+                                                                       g.gap_out);
+        break;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shared_vector(Glm &g)
+{
+    cudaError_t e = cudaMemsetAsync(g.v, 0, (size_t)g.dim * sizeof(float), g.stream);
+    if (e != cudaSuccess) return e;
+    k_shared_vector<<<(unsigned)g.sm_count * 8, kThreads, 0, g.stream>>>(g.indptr, g.indices, g.values, g.alpha,
+                                                                         g.n_coord, g.dim, g.v);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_refresh_resid(g);
+}
+
+} // namespace chicle

@@ -1,0 +1,257 @@
+"""GPU parity: the library, called through its C ABI, against the CPU oracle on the same seeded inputs.
+Integer results (partition, visiting orders) must be bit-exact; alpha, v and the gap within 1e-4 per round."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+from paper_1909_04885_b200 import binding, datagen  # noqa: E402
+from paper_1909_04885_b200.datagen import Phase, Workload  # noqa: E402
+
+import oracle  # noqa: E402
+from parity_util import check_partition, make_pair, rel_l2, run_parity, REL_TOL  # noqa: E402
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_1909_04885_b200 import build
+    build.build()
+    oracle.build()
+
+
+def tiny_dense(n, d, seed=0, loss="hinge", K=3, lam=None, rounds=4):
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((n, d)).astype(np.float32)
+    w = rng.standard_normal(d)
+    y = np.where(X @ w + 0.3 * rng.standard_normal(n) >= 0, 1.0, -1.0).astype(np.float32)
+    return Workload("tiny_dense", loss, "dense", n, d, X.reshape(-1), y, lam or 1.0 / n, rounds,
+                    [Phase(0, K, seed, float(K))])
+
+
+def tiny_csr(n, d, seed=0, loss="hinge", K=3, density=0.2, rounds=4, long_row=0, zero_rows=()):
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((n, d)).astype(np.float32)
+    X[rng.random((n, d)) > density] = 0.0
+    if long_row:
+        X[1, :long_row] = rng.standard_normal(long_row).astype(np.float32) * 0.1 + 0.5
+    for r in zero_rows:
+        X[r] = 0.0
+    w = rng.standard_normal(d)
+    y = np.where(X @ w >= 0, 1.0, -1.0).astype(np.float32)
+    indptr = np.zeros(n + 1, np.int64)
+    indptr[1:] = np.cumsum((X != 0).sum(1))
+    idx = np.nonzero(X)[1].astype(np.int32)
+    vals = X[X != 0].astype(np.float32)
+    return Workload("tiny_csr", loss, "csr", n, d, vals, y, 1.0 / n, rounds, [Phase(0, K, seed, float(K))], indptr, idx)
+
+
+# ------------------------------------------------------------------ a1, a2: integers, bit-exact
+@pytest.mark.parametrize("n,K,seed", [(10, 3, 0), (4096, 16, 1), (3 * 4096 + 17, 5, 2), (1000, 1, 3), (257, 257, 4),
+                                      (70000, 300, 5), (200003, 64, 2**63 + 11)])
+def test_partition_and_orders_bit_exact(n, K, seed):
+    w = tiny_dense(n, 4, seed=1, K=K)
+    w.phases = [Phase(0, K, seed, float(K))]
+    orc, glm = make_pair(w)
+    try:
+        orc.partition(K, seed)
+        glm.partition(K, seed)
+        check_partition(orc, glm, perm_rounds=(0, 3, 2**20 + 1))
+        # repartition with another K and seed (elastic K between rounds)
+        K2 = max(1, K // 2)
+        orc.partition(K2, seed + 1)
+        glm.partition(K2, seed + 1)
+        check_partition(orc, glm, perm_rounds=(1,))
+    finally:
+        glm.close()
+
+
+# ------------------------------------------------------------------ the five configurations
+def test_config1_hinge_dense_full():
+    run_parity(datagen.make("hinge_dense", 1))
+
+
+def test_config2_hinge_csr_scaled():
+    run_parity(datagen.make("hinge_csr", 100))
+
+
+def test_config3_logistic_dense_scaled():
+    run_parity(datagen.make("logistic_dense", 100))
+
+
+def test_config4_hinge_hashed_elastic_scaled():
+    w = datagen.make("hinge_hashed", 1000)
+    assert [p.K for p in w.phases] == [64, 16]
+    run_parity(w)
+
+
+def test_config5_ridge_csc_scaled():
+    run_parity(datagen.make("ridge_csc", 100))
+
+
+def test_config2_full_size_three_rounds():
+    # the benchmark's workload and launch configuration, element by element against the oracle
+    w = datagen.make("hinge_csr", 1)
+    run_parity(w, rounds=3, check_perm=True, on_device=True)
+
+
+def test_config3_full_size_two_rounds():
+    w = datagen.make("logistic_dense", 1)
+    run_parity(w, rounds=2, check_perm=False, on_device=True)
+
+
+# ------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("loss", ["hinge", "logistic"])
+@pytest.mark.parametrize("d", [1, 7, 28, 100, 1000])
+def test_dense_shapes(loss, d):
+    run_parity(tiny_dense(500, d, seed=d, loss=loss, K=4))
+
+
+@pytest.mark.parametrize("loss", ["hinge", "logistic"])
+def test_csr_with_zero_rows_and_a_row_longer_than_a_slot(loss):
+    run_parity(tiny_csr(300, 400, seed=7, loss=loss, K=4, density=0.05, long_row=300, zero_rows=(0, 17)))
+
+
+def test_single_partition_and_one_coordinate_per_partition():
+    run_parity(tiny_csr(64, 40, seed=3, K=1))
+    run_parity(tiny_csr(64, 40, seed=3, K=64))
+    run_parity(tiny_dense(50, 5, seed=3, K=50))
+
+
+@pytest.mark.parametrize("H", [1, 10, 37, 60, 250])
+def test_partial_and_multi_epoch_H(H):
+    # n_k = 25: H below, equal-ish and several local epochs
+    run_parity(tiny_dense(100, 6, seed=5, K=4), H=H)
+    run_parity(tiny_csr(100, 30, seed=5, K=4), H=H)
+
+
+def test_ridge_small_with_long_and_empty_columns():
+    rng = np.random.default_rng(11)
+    n, d = 300, 500
+    X = rng.random((n, d)).astype(np.float32)
+    X[rng.random((n, d)) > 0.1] = 0.0
+    X[:, 3] = rng.random(n).astype(np.float32) + 0.1      # a column longer than a slot
+    X[:, 9] = 0.0                                          # an empty column
+    w = np.zeros(d)
+    w[rng.choice(d, 20, replace=False)] = rng.standard_normal(20)
+    y = (X @ w + 0.01 * rng.standard_normal(n)).astype(np.float32)
+    XT = np.ascontiguousarray(X.T)
+    indptr = np.zeros(d + 1, np.int64)
+    indptr[1:] = np.cumsum((XT != 0).sum(1))
+    wl = Workload("ridge_tiny", "ridge", "csc", n, d, XT[XT != 0].astype(np.float32), y, 1e-2, 6,
+                  [Phase(0, 8, 0, 8.0)], indptr, np.nonzero(XT)[1].astype(np.int32))
+    run_parity(wl)
+
+
+def test_resync_mode_and_recomputed_shared_vector():
+    w = datagen.make("hinge_csr", 200)
+    run_parity(w, rounds=5, resync=True)
+    orc, glm = make_pair(w)
+    try:
+        orc.partition(4, 1)
+        glm.partition(4, 1)
+        for _ in range(2):
+            orc.cocoa_round(0, 4.0)
+        glm.set_state(orc.state.astype(np.float32), None, orc.round)      # v rebuilt on the device
+        assert rel_l2(glm.get_v(), orc.v) < 1e-5
+        assert glm.info()["round"] == 2
+        orc.cocoa_round(0, 4.0)
+        glm.cocoa_round(0, 4.0)
+        assert rel_l2(glm.get_alpha(), orc.state) < REL_TOL and rel_l2(glm.get_v(), orc.v) < REL_TOL
+    finally:
+        glm.close()
+
+
+def test_state_survives_repartition_bit_for_bit():
+    w = datagen.make("hinge_csr", 200)
+    orc, glm = make_pair(w)
+    try:
+        glm.partition(8, 0)
+        glm.cocoa_round(0, 8.0)
+        a0, v0, g0 = glm.get_alpha(), glm.get_v(), glm.duality_gap()
+        glm.partition(3, 5)
+        assert np.array_equal(a0, glm.get_alpha()) and np.array_equal(v0, glm.get_v())
+        assert glm.duality_gap() == g0 and glm.info()["round"] == 1
+    finally:
+        glm.close()
+
+
+def test_device_resident_inputs_and_plain_cuda_allocator_give_the_same_bits():
+    w = datagen.make("hinge_csr", 200)
+    res = []
+    for kw in ({}, {"on_device": True}, {"torch_allocator": False}):
+        glm = binding.from_workload(w, **kw)
+        glm.partition(4, 0)
+        for _ in range(3):
+            glm.cocoa_round(0, 4.0)
+        res.append((glm.get_alpha(), glm.get_v(), glm.duality_gap()["gap"]))
+        glm.close()
+    for r in res[1:]:
+        assert np.array_equal(r[0], res[0][0]) and np.array_equal(r[1], res[0][1]) and r[2] == res[0][2]
+
+
+def test_round_stats():
+    w = datagen.make("hinge_csr", 100)
+    glm = binding.from_workload(w)
+    try:
+        glm.partition(16, 0)
+        st = glm.cocoa_round(0, 16.0, stats=True)
+        assert st["steps"] == w.n_rows and st["ms_total"] > 0 and st["ms_local"] > 0
+        st = glm.cocoa_round(7, 16.0, stats=True)
+        assert st["steps"] == 7 * 16
+    finally:
+        glm.close()
+
+
+# ------------------------------------------------------------------ error behaviour
+def test_errors():
+    w = tiny_csr(50, 20, seed=1)
+    glm = binding.from_workload(w)
+    try:
+        with pytest.raises(binding.ChicleError) as e:
+            glm.cocoa_round(0, 1.0)
+        assert e.value.status == 2                                   # BAD_STATE: no partition yet
+        for K in (0, -1, 51):
+            with pytest.raises(binding.ChicleError) as e:
+                glm.partition(K, 0)
+            assert e.value.status == 1
+        glm.partition(2, 0)
+        for H, sp in ((-1, 1.0), (0, 0.0), (0, -2.0), (0, float("nan"))):
+            with pytest.raises(binding.ChicleError) as e:
+                glm.cocoa_round(H, sp)
+            assert e.value.status == 1
+        with pytest.raises(binding.ChicleError):
+            glm.get_permutation(0, 2, 25)
+        with pytest.raises(binding.ChicleError):
+            glm.get_permutation(0, 0, 24)
+        out = np.empty(49, np.float32)
+        with pytest.raises(binding.ChicleError):
+            glm._get(glm._lib.chicle_get_alpha, 49, out)
+        glm.cocoa_round(0, 2.0)                                      # the handle is still usable
+        assert glm.info()["round"] == 1
+    finally:
+        glm.close()
+    bad = tiny_csr(50, 20, seed=1)
+    bad.values = bad.values.copy()
+    bad.values[3] = np.nan
+    with pytest.raises(binding.ChicleError) as e:
+        binding.from_workload(bad)
+    assert e.value.status == 6
+    bad = tiny_csr(50, 20, seed=1)
+    bad.labels = bad.labels.copy()
+    bad.labels[4] = 0.5
+    with pytest.raises(binding.ChicleError) as e:
+        binding.from_workload(bad)
+    assert e.value.status == 1
+    bad = tiny_csr(50, 20, seed=1)
+    bad.indices = bad.indices.copy()
+    bad.indices[2] = 20
+    with pytest.raises(binding.ChicleError) as e:
+        binding.from_workload(bad)
+    assert e.value.status == 1
+    bad = tiny_csr(50, 20, seed=1)
+    bad.loss = "ridge"
+    with pytest.raises(binding.ChicleError) as e:
+        binding.from_workload(bad)
+    assert e.value.status == 5
