@@ -131,6 +131,20 @@ def aggregate(units_per_rank, world, seconds_max):
     return units_per_rank * world / seconds_max
 
 
+def read_traffic():
+    """DRAM bytes per local-solver launch from the committed ncu summary; None once the solver source has changed
+    since the counters were taken."""
+    import hashlib
+    try:
+        kv = dict(l.split() for l in open(os.path.join(ROOT, "profiles", "local_scd_traffic.txt")) if l.strip() and l[0] != "#")
+        src = open(os.path.join(ROOT, "paper_1909_04885_b200", "csrc", "solver.cu"), "rb").read()
+        if hashlib.sha256(src).hexdigest() != kv["solver_source_sha256"]:
+            return None
+        return int(kv["dram_bytes_per_launch"])
+    except Exception:
+        return None
+
+
 def time_oracle(w, ph, rounds_arg):
     """The oracle, untuned, on a bounded sample of the workload: whole rounds (+ gap) on min(K, cores) threads."""
     import oracle
@@ -271,13 +285,7 @@ def run_b200(args):
     ms_perm = statistics.mean(s["ms_permutation"] for s in stats)
     ms_red = statistics.mean(s["ms_reduce"] for s in stats)
     achieved = comp_bytes / (ms_local * 1e-3) / 1e9
-    traffic = None
-    prof = os.path.join(ROOT, "profiles", "local_scd_traffic.json")
-    if os.path.exists(prof) and args.scale == 1:
-        try:
-            traffic = json.load(open(prof)).get("dram_bytes_per_launch")
-        except Exception:
-            traffic = None
+    traffic = read_traffic() if args.scale == 1 else None
     owner_passes = 1 if ph.K <= 256 else 2
     launches = 1 + 5 * (8 + owner_passes) + 1 + 1 + 2   # order keys + radix passes, solver, aggregation, gap (2)
 
