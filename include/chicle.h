@@ -140,6 +140,34 @@ chicle_status_t chicle_set_state(chicle_glm_t *h, const float *host_alpha, const
 /* Current round counter, partition count and coordinate / shared-vector lengths; any pointer may be NULL. */
 chicle_status_t chicle_get_info(const chicle_glm_t *h, int64_t *round, int32_t *K, int64_t *n_coord, int64_t *dim);
 
+/* Largest problem chicle_partition_noalloc accepts: its workspace is a fixed array inside the library image. */
+#define CHICLE_NOALLOC_MAX_COORDS 131072
+
+/* The partition map of chicle_partition, for callers that must not allocate device memory. (The paper has no
+ * counterpart: this entry point exists for deployment reasons only.) Who needs it: code that asks for a partition
+ * map from a place where the device allocator is off limits, e.g. a serving or real-time loop whose memory pool was
+ * sized and frozen at start-up, a thread that holds a lock the allocator also wants, or a process whose device
+ * memory is handed out by another component. chicle_partition allocates its sort workspace and the K x dim update
+ * buffers; this call allocates nothing, on the host or on the device: no cudaMalloc, cudaFree, or framework
+ * allocator. Its workspace (about 3.2 MB) is a static device array that every GPU loading this library holds until
+ * the process ends.
+ *   device, cuda_stream   where to run; the work is enqueued on the stream and the call does not synchronise.
+ *   n_coord, K, seed      as in chicle_partition: 1 <= K <= n_coord <= CHICLE_NOALLOC_MAX_COORDS. A larger n_coord
+ *                         is refused with CHICLE_ERR_UNSUPPORTED and a message; nothing is launched.
+ *   dev_owner             out, device, n_coord int32: partition of every coordinate (what chicle_get_partition returns).
+ *   dev_members           out, device, n_coord int32: coordinate ids grouped by partition, ascending inside a partition;
+ *                         partition k occupies [off_k, off_{k+1}) with off_k = k*(n/K) + min(k, n mod K).
+ *   host_errbuf           optional host buffer of errbuf_len bytes that receives the error text (no handle exists to
+ *                         keep it). The caller owns both output arrays and the buffer.
+ * The first call on a device looks up the device address of the workspace (cudaGetSymbolAddress) and remembers it;
+ * make that first call outside any stream capture. All calls on a device share the one workspace, and it keeps
+ * whatever the previous call left in it; nothing in it needs clearing because every pass overwrites what it then
+ * reads. Two calls whose kernels overlap on the same GPU (different streams, or different host threads) race on it:
+ * serialise them. Results are bit-identical to chicle_partition's. */
+chicle_status_t chicle_partition_noalloc(int device, void *cuda_stream, int64_t n_coord, int32_t K, uint64_t seed,
+                                         int32_t *dev_owner, int32_t *dev_members, char *host_errbuf,
+                                         size_t errbuf_len);
+
 /* Text of the last error on this handle (library-owned, valid until the next call on the handle). With h = NULL:
  * the text of the last failed chicle_glm_create on this thread. Never NULL. */
 const char *chicle_last_error(const chicle_glm_t *h);

@@ -23,7 +23,7 @@ MEM_HOST, MEM_DEVICE = 0, 1
 
 EXPORTED = ["chicle_glm_create", "chicle_partition", "chicle_cocoa_round", "chicle_duality_gap", "chicle_get_alpha",
             "chicle_get_v", "chicle_get_partition", "chicle_get_permutation", "chicle_set_state", "chicle_get_info",
-            "chicle_last_error", "chicle_glm_destroy"]
+            "chicle_last_error", "chicle_glm_destroy", "chicle_partition_noalloc"]
 
 
 class ChicleError(RuntimeError):
@@ -87,6 +87,8 @@ def load():
     lib.chicle_last_error.argtypes = [vp]
     lib.chicle_glm_destroy.restype = None
     lib.chicle_glm_destroy.argtypes = [vp]
+    lib.chicle_partition_noalloc.restype = C.c_int
+    lib.chicle_partition_noalloc.argtypes = [C.c_int, vp, i64, i32, u64, vp, vp, C.c_char_p, C.c_size_t]
     _lib = lib
     return lib
 
@@ -267,3 +269,16 @@ def from_workload(w, device: int = 0, on_device: bool = False, **kw) -> Glm:
         indptr = None if indptr is None else torch.from_numpy(indptr).to(dev)
         indices = None if indices is None else torch.from_numpy(indices).to(dev)
     return Glm(w.loss, w.fmt, w.n_rows, w.n_cols, vals, labels, w.lam, indptr, indices, device=device, **kw)
+
+
+def partition_noalloc(n_coord: int, K: int, seed: int, owner_out, members_out, device: int = 0, stream: int = 0):
+    """``chicle_partition_noalloc``: fills two caller-owned int32 CUDA tensors of ``n_coord`` entries with the partition
+    map and the grouped member list, using the library's built-in workspace instead of allocating one. Meant for
+    callers that may not touch a device allocator at this point (frozen memory pools, serving loops). Asynchronous on
+    ``stream``; raises ``ChicleError`` with the library's message when the size is beyond the built-in limit."""
+    lib = load()
+    buf = C.create_string_buffer(256)
+    st = lib.chicle_partition_noalloc(device, C.c_void_p(stream), n_coord, K, C.c_uint64(seed & (2**64 - 1)),
+                                      C.c_void_p(owner_out.data_ptr()), C.c_void_p(members_out.data_ptr()), buf, 256)
+    if st != OK:
+        raise ChicleError(st, buf.value.decode())

@@ -1,5 +1,8 @@
 // Partition of the coordinates into K random equal blocks, and the per-round visiting orders.
 // Integer-only: the result is a pure function of (n, K, seed) and (seed, round, epoch).
+#include <cstdio>
+#include <mutex>
+
 #include "chicle_internal.cuh"
 
 namespace chicle {
@@ -115,3 +118,135 @@ cudaError_t launch_permutation(Glm &g, int64_t round, int64_t epochs)
 }
 
 } // namespace chicle
+
+namespace chicle {
+
+// ---------------------------------------------------------------------------------------------------------------
+// Partition without any allocation.
+//
+// Some callers are not allowed to allocate device memory when they need a partition map: code that runs inside a
+// region where the allocator must not be touched (a memory pool that was sized and frozen at start-up, a real-time
+// or serving loop with a fixed memory budget, a host thread that holds a lock the allocator also takes), or a
+// process whose device memory is handed out entirely by someone else. chicle_partition() cannot serve them: it
+// creates the sort workspace and the per-partition update buffers on its first call. The entry point below does
+// the same integer work (same kernels, same order, same result) with its workspace in a fixed array that is part
+// of the loaded library image, so no cudaMalloc, cudaFree or framework allocator is ever called.
+//
+// The array below is device memory owned by the CUDA module: every GPU that loads this library carries it until
+// the process exits. In host code its name is only a handle for the symbol, not an address a kernel may
+// dereference; the device address is fetched once per device with cudaGetSymbolAddress and that pointer is what
+// the kernels get.
+namespace {
+
+constexpr int64_t kNoAllocMaxCoords = CHICLE_NOALLOC_MAX_COORDS;
+constexpr size_t kNaKeysBytes = (size_t)kNoAllocMaxCoords * sizeof(uint64_t);                       // one key array
+constexpr size_t kNaValsBytes = (size_t)kNoAllocMaxCoords * sizeof(int32_t);                        // one id array
+constexpr size_t kNaHistBytes = (size_t)256 * ((kNoAllocMaxCoords + kSortTile - 1) / kSortTile) * sizeof(uint32_t);
+constexpr size_t kNaSumsBytes = 4096;                                                               // scan tile sums
+constexpr size_t kNaOffKeys0 = 0;
+constexpr size_t kNaOffKeys1 = kNaOffKeys0 + kNaKeysBytes;
+constexpr size_t kNaOffVals0 = kNaOffKeys1 + kNaKeysBytes;
+constexpr size_t kNaOffVals1 = kNaOffVals0 + kNaValsBytes;
+constexpr size_t kNaOffHist = kNaOffVals1 + kNaValsBytes;
+constexpr size_t kNaOffSums = kNaOffHist + kNaHistBytes;
+constexpr size_t kNaTotalBytes = kNaOffSums + kNaSumsBytes;
+static_assert(kNaKeysBytes % 256 == 0 && kNaValsBytes % 256 == 0 && kNaHistBytes % 256 == 0, "256-byte carving");
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaTotalBytes];
+
+constexpr int kNaMaxDevices = 64;
+std::mutex g_na_mutex;
+unsigned char *g_na_base[kNaMaxDevices] = {};
+
+void na_message(char *buf, size_t len, const char *msg)
+{
+    if (buf && len) std::snprintf(buf, len, "%s", msg);
+}
+
+} // namespace
+
+} // namespace chicle
+
+extern "C" chicle_status_t chicle_partition_noalloc(int device, void *cuda_stream, int64_t n_coord, int32_t K,
+                                                    uint64_t seed, int32_t *dev_owner, int32_t *dev_members,
+                                                    char *host_errbuf, size_t errbuf_len)
+{
+    using namespace chicle;
+    if (!dev_owner || !dev_members) {
+        na_message(host_errbuf, errbuf_len, "dev_owner and dev_members must be non-NULL device pointers");
+        return CHICLE_ERR_INVALID_ARG;
+    }
+    if (n_coord < 1 || n_coord > kNoAllocMaxCoords) {
+        na_message(host_errbuf, errbuf_len,
+                   "n_coord outside [1, CHICLE_NOALLOC_MAX_COORDS]: the built-in workspace holds at most 131072 "
+                   "coordinates; use chicle_partition for larger problems");
+        return CHICLE_ERR_UNSUPPORTED;
+    }
+    if (K < 1 || (int64_t)K > n_coord) {
+        na_message(host_errbuf, errbuf_len, "need 1 <= K <= n_coord");
+        return CHICLE_ERR_INVALID_ARG;
+    }
+    if (device < 0 || device >= kNaMaxDevices) {
+        na_message(host_errbuf, errbuf_len, "device index out of range");
+        return CHICLE_ERR_INVALID_ARG;
+    }
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        na_message(host_errbuf, errbuf_len, cudaGetErrorString(e));
+        return CHICLE_ERR_CUDA;
+    }
+    unsigned char *base = nullptr;
+    {
+        // set-up, once per device, with that device current: turn the symbol into a device address
+        std::lock_guard<std::mutex> lock(g_na_mutex);
+        if (!g_na_base[device]) {
+            void *p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+            if (e != cudaSuccess || !p) {
+                (void)cudaGetLastError();
+                na_message(host_errbuf, errbuf_len, e != cudaSuccess ? cudaGetErrorString(e) : "cudaGetSymbolAddress returned NULL");
+                return CHICLE_ERR_CUDA;
+            }
+            g_na_base[device] = static_cast<unsigned char *>(p);
+        }
+        base = g_na_base[device];
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint64_t *keys[2] = {reinterpret_cast<uint64_t *>(base + kNaOffKeys0), reinterpret_cast<uint64_t *>(base + kNaOffKeys1)};
+    int32_t *vals[2] = {reinterpret_cast<int32_t *>(base + kNaOffVals0), reinterpret_cast<int32_t *>(base + kNaOffVals1)};
+    uint32_t *hist = reinterpret_cast<uint32_t *>(base + kNaOffHist);
+    uint32_t *sums = reinterpret_cast<uint32_t *>(base + kNaOffSums);
+    // Nothing in the workspace has to start at zero: keys and ids are written before they are read, and every pass
+    // writes all of its digit counters and tile sums before scanning them, so the previous call's leftovers are
+    // never observed.
+    const int64_t n = n_coord;
+    const int T = 256;
+    k_partition_keys<<<blocks_for(n, T), T, 0, stream>>>(n, mix64(seed), keys[0], vals[0]);
+    int cur = 0;
+    for (int pass = 0; pass < 8; ++pass) {
+        e = radix_pass(keys[cur], vals[cur], keys[cur ^ 1], vals[cur ^ 1], nullptr, n, 8 * pass, hist, sums, stream);
+        if (e != cudaSuccess) break;
+        cur ^= 1;
+    }
+    if (e == cudaSuccess) {
+        k_owner_from_rank<<<blocks_for(n, T), T, 0, stream>>>(n, n / K, n % K, vals[cur], dev_owner);
+        k_iota<<<blocks_for(n, T), T, 0, stream>>>(n, vals[0]);
+        int passes = 1;
+        while (passes < 4 && (int64_t)K > (1LL << (8 * passes))) ++passes;
+        const int32_t *src = vals[0];
+        for (int p = 0; p < passes && e == cudaSuccess; ++p) {
+            int32_t *dst = p == passes - 1 ? dev_members : (src == vals[0] ? vals[1] : vals[0]);
+            e = radix_pass(nullptr, src, nullptr, dst, dev_owner, n, 8 * p, hist, sums, stream);
+            src = dst;
+        }
+    }
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        na_message(host_errbuf, errbuf_len, cudaGetErrorString(e));
+        return CHICLE_ERR_CUDA;
+    }
+    return CHICLE_OK;
+}
+
