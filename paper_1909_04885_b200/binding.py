@@ -13,7 +13,7 @@ from typing import Optional
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libchicle.so")
+LIB_PATH = os.environ.get("CHICLE_LIB_PATH") or os.path.join(_HERE, "libchicle.so")
 
 OK = 0
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_STATE", 3: "OOM", 4: "CUDA", 5: "UNSUPPORTED", 6: "NUMERIC", 7: "TIMEOUT"}
