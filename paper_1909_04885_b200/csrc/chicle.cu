@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in chicle.h: argument checks, the state machine, memory, and the order in
 // which the kernels of a round are enqueued. No arithmetic of the method happens here.
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -222,6 +223,41 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
         const std::string msg = h->err;
         return bail(st, msg);
     }
+    if (!dense) {
+        // frequency-rank the entry ids (see remap.cu); temporaries are released before returning
+        const int64_t dim = h->dim;
+        uint32_t *counts = nullptr, *hist = nullptr, *sums = nullptr;
+        uint64_t *keys[2] = {nullptr, nullptr};
+        int32_t *vals[2] = {nullptr, nullptr};
+        unsigned long long *mass = nullptr;
+        float *labels_new = nullptr;
+        bool ok2 = alloc_into(h, h->new_of_old, (size_t)dim) && alloc_into(h, h->old_of_new, (size_t)dim) &&
+                   alloc_into(h, h->perm_tmp, (size_t)dim) && alloc_into(h, counts, (size_t)dim) &&
+                   alloc_into(h, keys[0], (size_t)dim) && alloc_into(h, keys[1], (size_t)dim) &&
+                   alloc_into(h, vals[0], (size_t)dim) && alloc_into(h, vals[1], (size_t)dim) &&
+                   alloc_into(h, hist, sort_hist_entries(dim)) && alloc_into(h, sums, sort_scan_tiles(dim) + 1) &&
+                   alloc_into(h, mass, 4);
+        if (ok2 && ridge) ok2 = alloc_into(h, labels_new, (size_t)dim);
+        if (!ok2) return bail(CHICLE_ERR_OOM, "device allocation failed (id ranking)");
+        e = cudaMemsetAsync(counts, 0, (size_t)dim * 4, s);
+        if (e == cudaSuccess) e = cudaMemsetAsync(mass, 0, 32, s);
+        if (e == cudaSuccess) e = launch_frequency_remap(*h, counts, keys, vals, hist, sums, blocked_solver_hot_ids(), mass);
+        if (e == cudaSuccess && ridge) e = launch_gather_f32(*h, h->labels, h->old_of_new, dim, labels_new);
+        unsigned long long host_mass = 0;
+        if (e == cudaSuccess) e = cudaMemcpyAsync(&host_mass, mass, 8, cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) return bail_cuda(e, "id ranking kernels");
+        if (ridge) {
+            dev_free(h, h->labels);
+            h->labels = labels_new;
+        }
+        dev_free(h, counts); dev_free(h, keys[0]); dev_free(h, keys[1]); dev_free(h, vals[0]); dev_free(h, vals[1]);
+        dev_free(h, hist); dev_free(h, sums); dev_free(h, mass);
+        h->hot_variant = h->nnz > 0 && (double)host_mass >= 0.5 * (double)h->nnz ? 1 : 0;
+        const char *force = getenv("CHICLE_FORCE_VARIANT"); // debugging aid
+        if (force && strcmp(force, "flat") == 0) h->hot_variant = 0;
+        if (force && strcmp(force, "hot") == 0) h->hot_variant = 1;
+    }
     e = launch_sqnorm(*h);
     if (e == cudaSuccess) e = launch_refresh_resid(*h);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
@@ -390,6 +426,14 @@ chicle_status_t chicle_get_alpha(chicle_glm_t *h, float *out, int64_t len, chicl
 
 chicle_status_t chicle_get_v(chicle_glm_t *h, float *out, int64_t len, chicle_memspace_t space)
 {
+    if (h && h->new_of_old) {
+        // translate from the library's ranked ids to the caller's: tmp[old] = v[new_of_old[old]]
+        if (cudaSetDevice(h->device) == cudaSuccess) {
+            const cudaError_t e = launch_gather_f32(*h, h->v, h->new_of_old, h->dim, h->perm_tmp);
+            if (e != cudaSuccess) return fail_cuda(h, e, "chicle_get_v");
+        }
+        return copy_out(h, h->perm_tmp, h->dim, out, len, space, "chicle_get_v");
+    }
     return copy_out(h, h ? h->v : nullptr, h ? h->dim : 0, out, len, space, "chicle_get_v");
 }
 
@@ -429,7 +473,13 @@ chicle_status_t chicle_set_state(chicle_glm_t *h, const float *host_alpha, const
     if (e == cudaSuccess) e = cudaMemcpyAsync(h->alpha, host_alpha, (size_t)h->n_coord * 4, cudaMemcpyHostToDevice, h->stream);
     if (e == cudaSuccess) {
         if (host_v) {
-            e = cudaMemcpyAsync(h->v, host_v, (size_t)h->dim * 4, cudaMemcpyHostToDevice, h->stream);
+            if (h->new_of_old) {
+                // the caller's ids -> ranked ids: v[new] = host_v[old_of_new[new]]
+                e = cudaMemcpyAsync(h->perm_tmp, host_v, (size_t)h->dim * 4, cudaMemcpyHostToDevice, h->stream);
+                if (e == cudaSuccess) e = launch_gather_f32(*h, h->perm_tmp, h->old_of_new, h->dim, h->v);
+            } else {
+                e = cudaMemcpyAsync(h->v, host_v, (size_t)h->dim * 4, cudaMemcpyHostToDevice, h->stream);
+            }
             if (e == cudaSuccess) e = launch_refresh_resid(*h);
         } else {
             e = launch_shared_vector(*h);

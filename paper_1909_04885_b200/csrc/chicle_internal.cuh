@@ -74,6 +74,11 @@ struct Glm {
     float *alpha = nullptr;  // per coordinate: signed dual variable, or w for ridge
     float *v = nullptr;      // shared vector, dim
     float *resid = nullptr;  // ridge only: v - y, refreshed by the reduction kernel
+    // sparse problems: entry ids (positions in v) are frequency-ranked inside the library
+    int32_t *new_of_old = nullptr; // dim; nullptr when ids are not remapped (dense)
+    int32_t *old_of_new = nullptr; // dim
+    float *perm_tmp = nullptr;     // dim, staging for translating v at the boundary
+    int hot_variant = 0;           // 1: most non-zeros fall on the first ids, the solver keeps those in a direct array
 
     // partition
     int32_t K = 0;
@@ -112,5 +117,9 @@ cudaError_t launch_reduce(Glm &g);                                        // v +
 cudaError_t launch_gap(Glm &g);                                           // fills gap_out[0..2]
 cudaError_t launch_shared_vector(Glm &g);                                 // v = X^T alpha (or X w) from scratch
 cudaError_t launch_refresh_resid(Glm &g);                                 // ridge: resid = v - y
+cudaError_t launch_frequency_remap(Glm &g, uint32_t *counts, uint64_t *keys[2], int32_t *vals[2], uint32_t *hist,
+                                   uint32_t *scan_sums, int64_t hot_ids, unsigned long long *mass);
+cudaError_t launch_gather_f32(Glm &g, const float *src, const int32_t *map, int64_t n, float *dst); // dst[i] = src[map[i]]
+int blocked_solver_hot_ids();
 
 } // namespace chicle

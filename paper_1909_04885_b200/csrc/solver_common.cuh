@@ -11,14 +11,63 @@ namespace chicle {
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kNewtonIters = 5;
 
-struct SlotHdr {
+// Per-step header prepared by the staging warps. 48 bytes, 16-byte aligned, so that the chain reads it with two
+// 128-bit shared-memory loads: {row_start, coord, nnz} and {p0, p1, p2, p3}.
+struct alignas(16) SlotHdr {
     int64_t row_start;
     int32_t coord;
     int32_t nnz;
     float p0, p1, p2, p3;
-    int32_t pad[2];
+    int32_t pad[4];
 };
-static_assert(sizeof(SlotHdr) == 40 || sizeof(SlotHdr) == 48, "header size");
+static_assert(sizeof(SlotHdr) == 48, "header size");
+
+// Explicit shared-memory accesses with 32-bit addresses. The chain's loops are latency-bound; generic-address
+// loads through pointers the compiler cannot prove to be shared cost several times more per access.
+__device__ __forceinline__ float lds_f32(uint32_t a)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a)
+{
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 lds_f32x4(uint32_t a)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ int4 lds_s32x4(uint32_t a)
+{
+    int4 v;
+    asm volatile("ld.shared.v4.s32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t a, float v)
+{
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
+}
+
+// Sum over the warp through a 32-float shared-memory buffer: every lane stores its partial, then reads all 32 with
+// eight 128-bit loads and adds them in a fixed tree. About 100 cycles against about 150 for five shuffle rounds.
+// `buf` must be 16-byte aligned; the caller separates successive uses with __syncwarp().
+__device__ __forceinline__ float warp_sum_smem(float x, uint32_t buf, int lane)
+{
+    sts_f32(buf + 4u * lane, x);
+    __syncwarp();
+    const float4 a0 = lds_f32x4(buf), a1 = lds_f32x4(buf + 16), a2 = lds_f32x4(buf + 32), a3 = lds_f32x4(buf + 48);
+    const float4 a4 = lds_f32x4(buf + 64), a5 = lds_f32x4(buf + 80), a6 = lds_f32x4(buf + 96), a7 = lds_f32x4(buf + 112);
+    const float s0 = (a0.x + a0.y) + (a0.z + a0.w), s1 = (a1.x + a1.y) + (a1.z + a1.w);
+    const float s2 = (a2.x + a2.y) + (a2.z + a2.w), s3 = (a3.x + a3.y) + (a3.z + a3.w);
+    const float s4 = (a4.x + a4.y) + (a4.z + a4.w), s5 = (a5.x + a5.y) + (a5.z + a5.w);
+    const float s6 = (a6.x + a6.y) + (a6.z + a6.w), s7 = (a7.x + a7.y) + (a7.z + a7.w);
+    return ((s0 + s1) + (s2 + s3)) + ((s4 + s5) + (s6 + s7));
+}
 
 struct SolverParams {
     const int64_t *indptr;
@@ -70,16 +119,27 @@ __device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar)
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
-// Bounded wait. Returns false when the CTA is aborting (this wait or another one ran out).
+// Bounded wait for a whole warp (every lane must call it). Lane 0 polls, backing off with nanosleep so that waiting
+// warps do not crowd the shared-memory pipeline that the latency-bound chain warp depends on; the others are parked
+// at the warp barrier. Returns false when the CTA is aborting (this wait or another one ran out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status)
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 31u) == 31u && *abort_flag) return false;
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+        ok = 0;
+        for (uint32_t it = 0; it < kSpinLimit; ++it) {
+            if (mbar_try_wait(bar, parity)) { ok = 1; break; }
+            if (it >= 2) __nanosleep(it < 64 ? 32 : 256);
+            if ((it & 31u) == 31u && *abort_flag) break;
+        }
+        if (!ok && !*abort_flag) {
+            *abort_flag = 1;
+            atomicOr(status, ST_WAIT_TIMEOUT);
+        }
     }
-    *abort_flag = 1;
-    atomicOr(status, ST_WAIT_TIMEOUT);
-    return false;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();
+    return ok != 0;
 }
 
 __device__ __forceinline__ float warp_sum(float x)
