@@ -177,11 +177,13 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
     };
 
     const size_t nvals = dense ? (size_t)h->n_coord * (size_t)h->dim : (size_t)h->nnz;
-    bool ok = alloc_into(h, h->values, nvals) && alloc_into(h, h->labels, (size_t)h->n_examples) &&
+    // 4 spare elements behind values and indices: the solver's 16-byte bulk copies of a coordinate may read up to
+    // 12 bytes past its last entry
+    bool ok = alloc_into(h, h->values, nvals + 4) && alloc_into(h, h->labels, (size_t)h->n_examples) &&
               alloc_into(h, h->sqnorm, (size_t)h->n_coord) && alloc_into(h, h->alpha, (size_t)h->n_coord) &&
               alloc_into(h, h->v, (size_t)h->dim) && alloc_into(h, h->d_status, 64) &&
               alloc_into(h, h->gap_out, 8);
-    if (ok && !dense) ok = alloc_into(h, h->indptr, (size_t)h->n_coord + 1) && alloc_into(h, h->indices, nvals);
+    if (ok && !dense) ok = alloc_into(h, h->indptr, (size_t)h->n_coord + 1) && alloc_into(h, h->indices, nvals + 4);
     if (ok && ridge) ok = alloc_into(h, h->resid, (size_t)h->dim);
     h->gap_blocks = h->sm_count * 8;
     if (ok) ok = alloc_into(h, h->gap_partials, (size_t)h->gap_blocks * 4);

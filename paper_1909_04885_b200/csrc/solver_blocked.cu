@@ -2,28 +2,35 @@
 // walked strictly in order (paper Sec. 2.1 worker structure with L = 1; Sec. 5.1: SCD local solver), with the
 // part of the local model that the next steps can touch held in shared memory.
 //
-// Local model: v_local = v + sigma' * U_k; U_k (the partition's accumulated update, zero at round start) has its
-// home in row k of the K x dim workspace in global memory. Entry ids are frequency-ranked when the problem is
-// created (id 0 is the most frequent feature), which gives two places for the live part of U_k:
-//   hot   ids below HOT: a direct array in shared memory for the whole kernel (no look-up at all);
+// Local model: w_local = v + sigma' * U_k, where U_k (the partition's accumulated update, zero at round start) has
+// its home in row k of the K x dim workspace in global memory. Shared memory holds w_local itself at the entries
+// that matter, so a step is one gather, one reduction, the scalar step and one scatter (w_local += sigma' delta x);
+// U_k is recovered as (w_local - v) / sigma' when an entry leaves shared memory. Entry ids are frequency-ranked when
+// the problem is created (id 0 is the most frequent feature), which gives two places for the live part:
+//   hot   ids below HOT: a direct array for the whole kernel (no look-up at all);
 //   cold  the remaining ids: the walk is cut into blocks of kB consecutive steps and, per block, the helper warps
-//         build a small open-addressing hash table in shared memory over the block's distinct cold ids.
-// Every staged non-zero carries its value, the read-only v at its id (gathered by the helpers with cp.async; v is
-// constant during a round) and a 16-bit slot (hot id, or HOT + table slot). The chain warp runs a block's steps
-// entirely against shared memory: gather, butterfly reduction, scalar step in registers, scatter.
+//         build a small open-addressing hash table over the block's distinct cold ids.
+// Every staged non-zero carries its value and a 16-bit index into the shared array (hot id, or table slot).
 //
-// A cold slot's U_k value comes from the previous block's table when that block touches the id too ("carried":
-// copied shared-to-shared once the chain has finished the previous block) and from global memory otherwise,
-// fetched early while the chain is still busy (the id is not in the previous block, so its global value is final:
-// older blocks were written back before). A finished block's table goes back to global memory off the critical
-// path, and so do the new alpha values, which the chain parks in the block's headers. The result equals walking
-// the coordinates one by one against a full copy of the local model.
+// A cold slot's value comes from the previous block's table when that block touches the id too ("carried": copied
+// shared-to-shared once the chain has finished the previous block) and from global memory otherwise, fetched early
+// while the chain is still busy (the id is not in the previous block, so its global value is final: older blocks
+// were written back before). A finished block's table goes back to global memory off the critical path, and so do
+// the new alpha values, which the chain parks in the block's headers. The result equals walking the coordinates
+// one by one against a full copy of the local model, up to rounding.
+//
+// The chain warp's loop is latency-bound and shares the SM with the helpers, and measurements showed that what
+// slows it is load/store-unit traffic from the other warps (4-byte cp.async or plain global loads at a high rate
+// made a step five times slower), not their arithmetic or their shared-memory atomics. Hence: the non-zeros of a
+// coordinate arrive by bulk copies of the copy engine (16-byte aligned windows around the coordinate, one
+// instruction per array), v is folded into the shared array instead of being gathered per non-zero, the roles hand
+// blocks over through named hardware barriers (no polling), and the chain uses explicit 32-bit shared addresses.
 //
 // Staging runs three blocks deep: visiting-order entries three blocks ahead, per-coordinate fields two blocks
-// ahead (one helper warp does nothing else), non-zeros one block ahead (cp.async into a staging area). A block that
-// does not fit (a coordinate longer than CAP, too many distinct cold ids) is walked by the chain against global
-// memory for its cold ids. The roles hand blocks over through named hardware barriers (no polling); every role
-// runs the same number of blocks and leaves only at the end, so each barrier always gets its full count.
+// ahead (one helper warp does nothing else), non-zeros one block ahead. A block that does not fit (a coordinate
+// longer than CAP, too many distinct cold ids) is walked by the chain against global memory for its cold ids.
+// Every role runs the same number of blocks and leaves only at the end, so each barrier always gets its full count;
+// the one polled wait (for the bulk copies) is bounded.
 #include "solver_common.cuh"
 
 namespace chicle {
@@ -44,27 +51,30 @@ constexpr uint16_t kNoCarry = 0xFFFFu;
 template <int HTC, int CAP> struct BlockBuf {
     SlotHdr hdr[kB];
     float val[kB][CAP];
-    float vb[kB][CAP];      // v at the entry's id
-    int32_t key[HTC];
-    uint16_t pos[kB][CAP];  // index into the U array: hot id, or the block's table slot behind the hot ids
+    int32_t key[HTC];       // cold id in a table slot, -1 = empty
+    float Tv[HTC];          // v at that id (to turn w_local back into U_k)
+    uint16_t pos[kB][CAP];  // index into the W array: hot id, or this buffer's table slot behind the hot ids
     uint16_t occ[HTC];      // occupied table slots, in insertion order
     uint16_t carry[HTC];    // slot of the same id in the previous block's table, or kNoCarry
     int32_t n_occ, cnt, slow, pad;
 };
 
 template <int CAP> struct Stage {
-    int32_t idx[kB][CAP];
-    float val[kB][CAP];
-    uint16_t cold[kB * CAP]; // (coordinate << 8 | entry) of the staged block's cold non-zeros
-    SlotHdr hdr[2][kB];      // headers of the block being built and of the next one
+    // Rows are 16-byte aligned windows of the global arrays: coordinate j's entry e sits at [j][shift[j] + e].
+    alignas(16) int32_t idx[kB][CAP + 4];
+    alignas(16) float val[kB][CAP + 4];
+    alignas(8) uint64_t bar;  // counts the bytes of the bulk copies of the block being staged
+    uint16_t cold[kB * CAP];  // (coordinate << 8 | entry) of the staged block's cold non-zeros
+    SlotHdr hdr[2][kB];       // headers of the block being built and of the next one
+    int32_t shift[2][kB];
     int32_t cnt[2], slow[2];
-    int32_t n_cold, pad;
+    int32_t n_cold, abort_flag;
 };
 
 template <int HOT, int HTC, int CAP> struct SharedB {
-    // U_k in shared memory, one array so that the chain needs no case split: [0, HOT) the hot ids, then the cold
-    // table of buffer 0, then the cold table of buffer 1
-    alignas(16) float U[HOT + 2 * HTC];
+    // w_local in shared memory, one array so that the chain needs no case split: [0, HOT) the hot ids, then the
+    // cold table of buffer 0, then the cold table of buffer 1
+    alignas(16) float W[HOT + 2 * HTC + 32]; // + one dummy word per chain lane (always 0)
     alignas(16) float red[32]; // the chain's reduction buffer
     Stage<CAP> st;
     BlockBuf<HTC, CAP> buf[2];
@@ -72,8 +82,7 @@ template <int HOT, int HTC, int CAP> struct SharedB {
 
 // Named hardware barriers. 1: among the helpers. 2 ("done"): the chain arrives when it has finished a block, the
 // helpers wait. 3 ("full"): the helpers arrive when a block is ready, the chain waits. Blocking on a hardware
-// barrier costs no issue slots and no shared-memory traffic, which matters because the chain's latency-bound loop
-// shares the SM with the waiters (polling an mbarrier from 7 warps tripled the chain's step time).
+// barrier costs no issue slots and no shared-memory traffic.
 __device__ __forceinline__ void helper_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kHelperThreads) : "memory"); }
 __device__ __forceinline__ void done_arrive() { __threadfence_block(); asm volatile("bar.arrive 2, %0;" ::"n"(kThreadsB) : "memory"); }
 __device__ __forceinline__ void done_wait() { asm volatile("bar.sync 2, %0;" ::"n"(kThreadsB) : "memory"); }
@@ -95,16 +104,62 @@ template <int LOSS> __device__ __forceinline__ void refresh_state(SlotHdr &h, co
     h.p1 = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? al : h.p3 * al;
 }
 
+// What the chain keeps in registers for one step: header fields, and per 32-lane chunk of the coordinate this
+// lane's value and the shared address of its w_local word (the lane's dummy word beyond the coordinate's length).
+template <int CHUNKS> struct StepRegs {
+    float4 p;
+    int32_t coord, nnz;
+    float x[CHUNKS];
+    uint32_t wa[CHUNKS];
+};
+
+// The loads of a step's header, slots and values, as issued (nothing here waits for a result) ...
+template <int CHUNKS> struct StepRaw {
+    int4 hi;
+    float4 p;
+    uint32_t s[CHUNKS];
+    float x[CHUNKS];
+};
+template <int CHUNKS, int CAP>
+__device__ __forceinline__ void issue_step(StepRaw<CHUNKS> &r, int j, uint32_t hdr0, uint32_t pos0, uint32_t val0)
+{
+    const uint32_t hb = hdr0 + 48u * j;
+    r.hi = lds_s32x4(hb);
+    r.p = lds_f32x4(hb + 16);
+    const uint32_t pb = pos0 + (uint32_t)(2 * CAP) * j, xb = val0 + (uint32_t)(4 * CAP) * j;
+#pragma unroll
+    for (int c = 0; c < CHUNKS; ++c) {
+        r.s[c] = lds_u16(pb + 64u * c); // always a valid shared address; the content counts only if active
+        r.x[c] = lds_f32(xb + 128u * c);
+    }
+}
+// ... and their first use, placed where the results have long arrived.
+template <int CHUNKS>
+__device__ __forceinline__ void finish_step(StepRegs<CHUNKS> &r, const StepRaw<CHUNKS> &raw, uint32_t wbase, uint32_t dummy,
+                                            int lane)
+{
+    r.p = raw.p;
+    r.coord = raw.hi.z;
+    r.nnz = raw.hi.w;
+#pragma unroll
+    for (int c = 0; c < CHUNKS; ++c) {
+        const bool active = lane + 32 * c < r.nnz;
+        r.wa[c] = wbase + 4u * (active ? raw.s[c] : dummy);
+        r.x[c] = active ? raw.x[c] : 0.0f;
+    }
+}
+
 template <int LOSS, int HOT, int HTC, int CAP>
 __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const SolverParams P)
 {
-    static_assert((HTC & (HTC - 1)) == 0 && HOT + 2 * HTC <= 65535 && CAP % 32 == 0 && CAP <= 256, "slot encoding");
+    static_assert((HTC & (HTC - 1)) == 0 && HOT + 2 * HTC + 32 <= 65535 && CAP % 32 == 0 && CAP <= 252, "slot encoding");
     using Shared = SharedB<HOT, HTC, CAP>;
     using Buf = BlockBuf<HTC, CAP>;
     constexpr int kMaxOcc = HTC * 3 / 4; // distinct cold ids a block may have before it is walked unstaged
     constexpr int kChunks = CAP / 32;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Shared &sh = *reinterpret_cast<Shared *>(smem_raw);
+    Stage<CAP> &st = sh.st;
     const int k = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -112,75 +167,86 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
     const int64_t nk = P.part_off[k + 1] - off;
     const int64_t steps = nk <= 0 ? 0 : (P.H == 0 ? nk : P.H);
     float *Uk = P.U + (size_t)k * (size_t)P.dim;
-    const int hot_n = HOT < P.dim ? HOT : (int)P.dim; // ids below hot_n live in Uhot
-    for (int i = threadIdx.x; i < hot_n; i += kThreadsB) sh.U[i] = Uk[i];
+    const int hot_n = HOT < P.dim ? HOT : (int)P.dim; // ids below hot_n live in the direct part of W
+    const float inv_sigma = 1.0f / P.sigma;
+    if (threadIdx.x == 0) {
+        st.abort_flag = 0;
+        mbar_init(smem_u32(&st.bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); // make the init visible to the copy engine
+    }
+    for (int i = threadIdx.x; i < hot_n; i += kThreadsB) sh.W[i] = fmaf(P.sigma, Uk[i], P.vbase[i]);
+    if (threadIdx.x < 32) sh.W[HOT + 2 * HTC + threadIdx.x] = 0.0f;
     __syncthreads();
     if (steps == 0) return;
     const int64_t nblocks = (steps + kB - 1) / kB;
 
     if (warp == 0) {
         // =============================== the chain ===============================
-        const uint32_t ubase = smem_u32(&sh.U[0]);
+        const uint32_t wbase = smem_u32(&sh.W[0]);
         const uint32_t redbuf = smem_u32(&sh.red[0]);
+        const uint32_t dummy = HOT + 2 * HTC + lane; // this lane's dummy word in W
+        const float sigma = P.sigma;
         for (int64_t b = 0; b < nblocks; ++b) {
             Buf &B = sh.buf[b & 1];
             full_wait();
             const int cnt = B.cnt;
             const bool staged = B.slow == 0;
-            for (int j = 0; j < cnt; ++j) {
-                const uint32_t hb = smem_u32(&B.hdr[j]);
-                SlotHdr h;
-                {
-                    const int4 hi = lds_s32x4(hb);
-                    const float4 hp = lds_f32x4(hb + 16);
-                    h.row_start = ((int64_t)hi.y << 32) | (uint32_t)hi.x;
-                    h.coord = hi.z;
-                    h.nnz = hi.w;
-                    h.p0 = hp.x; h.p1 = hp.y; h.p2 = hp.z; h.p3 = hp.w;
-                }
-                if (P.multi_epoch) refresh_state<LOSS>(h, P.alpha, lane);
-                float acc = 0.0f, delta, new_state;
-                if (staged) {
-                    // all of the coordinate's entries in registers: the loads go out back to back
-                    const uint32_t pb = smem_u32(&B.pos[j][0]) + 2u * lane;
-                    const uint32_t xb = smem_u32(&B.val[j][0]) + 4u * lane;
-                    const uint32_t vb = smem_u32(&B.vb[j][0]) + 4u * lane;
-                    float x[kChunks], u[kChunks];
-                    uint32_t ua[kChunks];
+            if (staged) {
+                // Branch-free, software-pipelined walk: the next step's header, values and slots are loaded while
+                // this step's reduction runs (they do not depend on it); lanes beyond the coordinate's length are
+                // pointed at a private dummy word with value 0, so gather and scatter need no predicates.
+                const uint32_t hdr0 = smem_u32(&B.hdr[0]);
+                const uint32_t pos0 = smem_u32(&B.pos[0][0]) + 2u * lane;
+                const uint32_t val0 = smem_u32(&B.val[0][0]) + 4u * lane;
+                StepRegs<kChunks> cur;
+                StepRaw<kChunks> raw;
+                issue_step<kChunks, CAP>(raw, 0, hdr0, pos0, val0);
+                finish_step<kChunks>(cur, raw, wbase, dummy, lane);
+                for (int j = 0; j < cnt; ++j) {
+                    if (j + 1 < cnt) issue_step<kChunks, CAP>(raw, j + 1, hdr0, pos0, val0);
+                    SlotHdr h;
+                    h.row_start = 0;
+                    h.coord = cur.coord;
+                    h.nnz = cur.nnz;
+                    h.p0 = cur.p.x; h.p1 = cur.p.y; h.p2 = cur.p.z; h.p3 = cur.p.w;
+                    if (P.multi_epoch) refresh_state<LOSS>(h, P.alpha, lane);
+                    float w[kChunks];
+                    float acc = 0.0f, delta, new_state;
 #pragma unroll
                     for (int c = 0; c < kChunks; ++c) {
-                        x[c] = 0.0f;
-                        u[c] = 0.0f;
-                        ua[c] = 0xFFFFFFFFu;
-                        if (lane + 32 * c < h.nnz) {
-                            ua[c] = ubase + 4u * lds_u16(pb + 64u * c);
-                            x[c] = lds_f32(xb + 128u * c);
-                            const float vv = lds_f32(vb + 128u * c);
-                            u[c] = lds_f32(ua[c]);
-                            acc = fmaf(x[c], fmaf(P.sigma, u[c], vv), acc);
-                        }
+                        w[c] = lds_f32(cur.wa[c]);
+                        acc = fmaf(cur.x[c], w[c], acc);
                     }
                     acc = warp_sum_smem(acc, redbuf, lane);
                     coordinate_step<LOSS>(acc, h, delta, new_state);
-                    if (!(fabsf(delta) <= CUDART_MAX_NORMAL_F)) {
-                        if (lane == 0) atomicOr(P.status, ST_NONFINITE_STEP);
-                        delta = 0.0f;
-                        new_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? h.p1 : h.p3 * h.p1;
-                    }
-                    if (delta != 0.0f) {
+                    // (a non-finite step is caught off the chain, when the helpers write alpha out)
+                    if (delta != 0.0f) { // the same in every lane
+                        const float sd = sigma * delta;
 #pragma unroll
-                        for (int c = 0; c < kChunks; ++c)
-                            if (ua[c] != 0xFFFFFFFFu) sts_f32(ua[c], fmaf(delta, x[c], u[c]));
+                        for (int c = 0; c < kChunks; ++c) sts_f32(cur.wa[c], fmaf(sd, cur.x[c], w[c]));
                     }
-                } else {
-                    // unstaged block: hot ids from shared memory, cold ids straight from global memory (current
-                    // there: the helpers wrote the previous table back before handing this block over)
+                    if (lane == 0) {
+                        // parked in the header and written out by the helpers, off the chain, unless the round
+                        // revisits coordinates and needs it in place at once
+                        if (P.multi_epoch) P.alpha[h.coord] = new_state;
+                        else sts_f32(hdr0 + 48u * j + 20u, new_state); // the header's p1 field
+                    }
+                    __syncwarp();
+                    finish_step<kChunks>(cur, raw, wbase, dummy, lane);
+                }
+            } else {
+                // unstaged block: hot ids from shared memory, cold ids straight from global memory (current there:
+                // the helpers wrote the previous table back before handing this block over)
+                for (int j = 0; j < cnt; ++j) {
+                    SlotHdr h = B.hdr[j];
+                    if (P.multi_epoch) refresh_state<LOSS>(h, P.alpha, lane);
+                    float acc = 0.0f, delta, new_state;
                     const int32_t *ix = P.indices + h.row_start;
                     const float *xv = P.values + h.row_start;
                     for (int e = lane; e < h.nnz; e += 32) {
                         const int32_t i = ix[e];
-                        const float uu = i < hot_n ? sh.U[i] : Uk[i];
-                        acc = fmaf(xv[e], fmaf(P.sigma, uu, P.vbase[i]), acc);
+                        const float ww = i < hot_n ? sh.W[i] : fmaf(sigma, Uk[i], P.vbase[i]);
+                        acc = fmaf(xv[e], ww, acc);
                     }
                     acc = warp_sum(acc);
                     coordinate_step<LOSS>(acc, h, delta, new_state);
@@ -192,24 +258,19 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                     if (delta != 0.0f)
                         for (int e = lane; e < h.nnz; e += 32) {
                             const int32_t i = ix[e];
-                            if (i < hot_n) sh.U[i] = fmaf(delta, xv[e], sh.U[i]);
+                            if (i < hot_n) sh.W[i] = fmaf(sigma * delta, xv[e], sh.W[i]);
                             else Uk[i] = fmaf(delta, xv[e], Uk[i]);
                         }
+                    if (lane == 0) {
+                        if (P.multi_epoch) P.alpha[h.coord] = new_state;
+                        else B.hdr[j].p1 = new_state;
+                    }
+                    __syncwarp();
                 }
-                if (lane == 0) {
-                    // parked in the header and written out by the helpers, off the chain, unless the round revisits
-                    // coordinates and needs it in place at once
-                    if (P.multi_epoch) P.alpha[h.coord] = new_state;
-                    else sts_f32(hb + 20, new_state); // the header's p1 field
-                }
-                __syncwarp();
             }
             __syncwarp();
             done_arrive();
         }
-        // the hot part of U_k goes home
-        __syncwarp();
-        for (int i = lane; i < hot_n; i += 32) Uk[i] = sh.U[i];
         return;
     }
 
@@ -218,7 +279,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
     const bool hdr_warp = ht < 32;       // helper warp 0 prepares headers, the others stage non-zeros
     const int et = ht - 32;              // index among the entry-staging threads (valid when !hdr_warp)
     const int ew = et >> 5;
-    Stage<CAP> &st = sh.st;
+    volatile int *abort_flag = &st.abort_flag;
 
     // Header pipeline, in registers of the header warp: the coordinate of step `lane` of block b+3 is in flight,
     // the fields of block b+2 are in flight, block b+1's fields are turned into headers during iteration b.
@@ -265,24 +326,34 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
             }
             hd.pad[0] = hd.pad[1] = hd.pad[2] = hd.pad[3] = 0;
             st.hdr[q][lane] = hd;
+            st.shift[q][lane] = (int32_t)(f.rs & 3);
         }
         const bool too_long = __any_sync(0xffffffffu, nnz > CAP);
         if (lane == 0) {
             st.cnt[q] = cnt;
             st.slow[q] = too_long ? 1 : 0;
         }
+        return too_long;
     };
-    // entry warps only: cp.async of block `blk`'s non-zeros into the staging area
-    auto issue_entries = [&](int64_t blk) {
-        const int q = (int)(blk & 1);
-        if (st.slow[q]) return;
-        for (int j = ew; j < st.cnt[q]; j += kEntryWarps) {
-            const int nnz = st.hdr[q][j].nnz;
-            const int64_t rs = st.hdr[q][j].row_start;
-            for (int e = lane; e < nnz; e += 32) {
-                cp_async4(smem_u32(&st.idx[j][e]), P.indices + rs + e);
-                cp_async4(smem_u32(&st.val[j][e]), P.values + rs + e);
-            }
+    // header warp only: lane j starts the two bulk copies of coordinate j of the block whose fields are `f`
+    // (16-byte aligned windows: up to 3 elements before the coordinate and up to 3 behind it come along)
+    auto issue_entries = [&](const Fields &f, bool too_long) {
+        if (too_long) return;
+        uint32_t bytes = 0;
+        int64_t first = 0;
+        if (f.c >= 0 && f.re > f.rs) {
+            first = f.rs & ~(int64_t)3;
+            bytes = (uint32_t)(((f.re - first) + 3) & ~(int64_t)3) * 4u;
+        }
+        uint32_t total = 2u * bytes;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+        const uint32_t bar = smem_u32(&st.bar);
+        if (lane == 0) mbar_arrive_expect_tx(bar, total);
+        __syncwarp();
+        if (bytes) {
+            bulk_g2s(smem_u32(&st.idx[lane][0]), P.indices + first, bytes, bar);
+            bulk_g2s(smem_u32(&st.val[lane][0]), P.values + first, bytes, bar);
         }
     };
 
@@ -294,18 +365,19 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
         f_next = issue_fields(coord_of(1));
         f_far = issue_fields(coord_of(2));
         c_far = coord_of(3);
-        stage_headers(0, f0);
+        const bool too_long = stage_headers(0, f0);
+        issue_entries(f0, too_long);
     }
     helper_bar();
-    if (!hdr_warp) issue_entries(0);
 
     const uint32_t lt_mask = (1u << lane) - 1u;
+    uint32_t n_staged = 0; // blocks whose non-zeros came through the bulk-copy barrier so far (its phase counter)
     for (int64_t b = 0; b < nblocks; ++b) {
         const int q = (int)(b & 1);
         Buf &B = sh.buf[q];
         Buf &Prev = sh.buf[q ^ 1];
-        float *Tu = sh.U + HOT + q * HTC;          // this block's cold table values
-        float *TuPrev = sh.U + HOT + (q ^ 1) * HTC; // the previous block's
+        float *Tw = sh.W + HOT + q * HTC;          // this block's cold table: w_local at the slot's id
+        float *TwPrev = sh.W + HOT + (q ^ 1) * HTC; // the previous block's
         const bool have_prev = b > 0;
         // ---- S0: reset this buffer's table (its previous block was written back in the last iteration)
         for (int p = ht; p < HTC; p += kHelperThreads) B.key[p] = -1;
@@ -313,33 +385,41 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
             B.n_occ = 0;
             st.n_cold = 0;
         }
-        cp_async_wait_all();
-        helper_bar(); // the staging area holds block b's non-zeros; its headers are in st.hdr[q]
         const int cnt = st.cnt[q];
         bool slow = st.slow[q] != 0;
+        if (!slow) {
+            // the bulk copies of block b must have landed (bounded wait; lane 0 of each warp polls)
+            if (!mbar_wait(smem_u32(&st.bar), n_staged & 1u, abort_flag, P.status)) slow = true;
+            ++n_staged;
+        }
+        helper_bar(); // the staging area holds block b's non-zeros; its headers are in st.hdr[q]
+        if (*abort_flag) slow = true; // copies that never landed: walk the block unstaged (the status word has it)
         const bool prev_slow = have_prev && Prev.slow != 0;
         // cold ids that are not in the previous table may be fetched from global memory now, unless the chain is
         // writing global memory itself (previous block unstaged)
         const bool early_ok = !prev_slow;
+        bool next_too_long = false;
+        Fields f_issue{-1, 0, 0, 0.f, 0.f, 0.f};
         if (hdr_warp) {
             // ---- the header warp advances the header pipeline while the others build the table
             if (lane < cnt) B.hdr[lane] = st.hdr[q][lane];
-            if (b + 1 < nblocks) stage_headers(b + 1, f_next);
+            f_issue = f_next;
+            if (b + 1 < nblocks) next_too_long = stage_headers(b + 1, f_next);
             f_next = f_far;
             f_far = issue_fields(c_far);
             c_far = coord_of(b + 4);
         } else if (!slow) {
             // ---- S3a: classify. An entry warp takes whole coordinates, lanes over the non-zeros: copy the value,
-            //      start the gather of v, give hot ids their slot, collect cold ones in a list.
+            //      give hot ids their index, collect cold ones in a list.
             for (int j = ew; j < cnt; j += kEntryWarps) {
                 const int nnz = st.hdr[q][j].nnz;
+                const int sft = st.shift[q][j];
                 for (int e0 = 0; e0 < nnz; e0 += 32) {
                     const int e = e0 + lane;
                     bool cold = false;
                     if (e < nnz) {
-                        const int32_t idx = st.idx[j][e];
-                        B.val[j][e] = st.val[j][e];
-                        cp_async4(smem_u32(&B.vb[j][e]), P.vbase + idx);
+                        const int32_t idx = st.idx[j][sft + e];
+                        B.val[j][e] = st.val[j][sft + e];
                         if (HOT > 0 && idx < HOT) B.pos[j][e] = (uint16_t)idx;
                         else cold = true;
                     }
@@ -365,7 +445,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                 if (i < n_cold) {
                     const uint32_t je = st.cold[i];
                     const int j = je >> 8, e = je & 255;
-                    const int32_t idx = st.idx[j][e];
+                    const int32_t idx = st.idx[j][st.shift[q][j] + e];
                     p = hash_slot<HTC>(idx);
                     bool placed = false;
                     if (B.n_occ <= kMaxOcc) {
@@ -391,40 +471,58 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                 }
             }
         }
-        helper_bar(); // all slots known
+        helper_bar(); // all slots known; the staging area is free
+        // ---- S5: the header warp starts the bulk copies of block b+1 (its fields are in f_issue)
+        if (hdr_warp && b + 1 < nblocks) issue_entries(f_issue, next_too_long);
         if (!slow && (B.slow == 2 || B.n_occ > kMaxOcc)) slow = true;
         if (!slow) {
-            // ---- S3c: per distinct cold id, look it up in the previous table and fetch U_k if it is final
+            // ---- S3c: per distinct cold id: v, a look-up in the previous table, and w_local if U_k is final
             const int n_occ = B.n_occ;
-            for (int i = ht; i < n_occ; i += kHelperThreads) {
-                const uint32_t p = B.occ[i];
-                const int32_t idx = B.key[p];
-                uint16_t cp = kNoCarry;
-                if (have_prev && !prev_slow) {
-                    uint32_t r = hash_slot<HTC>(idx);
-                    for (int probe = 0; probe < HTC; ++probe) {
-                        const int32_t kr = Prev.key[r];
-                        if (kr == idx) { cp = (uint16_t)r; break; }
-                        if (kr == -1) break;
-                        r = (r + 1) & (HTC - 1);
+            for (int base = 0; base < n_occ; base += 2 * kHelperThreads) {
+                uint32_t pp[2];
+                float vv[2], uu[2];
+                bool fetch[2];
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const int i = base + r * kHelperThreads + ht;
+                    pp[r] = HTC;
+                    fetch[r] = false;
+                    vv[r] = uu[r] = 0.0f;
+                    if (i >= n_occ) continue;
+                    const uint32_t p = B.occ[i];
+                    const int32_t idx = B.key[p];
+                    uint16_t cp = kNoCarry;
+                    if (have_prev && !prev_slow) {
+                        uint32_t r2 = hash_slot<HTC>(idx);
+                        for (int probe = 0; probe < HTC; ++probe) {
+                            const int32_t kr = Prev.key[r2];
+                            if (kr == idx) { cp = (uint16_t)r2; break; }
+                            if (kr == -1) break;
+                            r2 = (r2 + 1) & (HTC - 1);
+                        }
                     }
+                    B.carry[p] = cp;
+                    pp[r] = p;
+                    vv[r] = P.vbase[idx];
+                    fetch[r] = cp == kNoCarry && early_ok;
+                    if (fetch[r]) uu[r] = Uk[idx]; // only this SM writes U_k, so a cached copy cannot be stale
                 }
-                B.carry[p] = cp;
-                // U_k is only ever written by this SM, so a cached copy cannot be stale
-                if (cp == kNoCarry && early_ok) cp_async4(smem_u32(&Tu[p]), Uk + idx);
+#pragma unroll
+                for (int r = 0; r < 2; ++r)
+                    if (pp[r] < HTC) {
+                        B.Tv[pp[r]] = vv[r];
+                        if (fetch[r]) Tw[pp[r]] = fmaf(P.sigma, uu[r], vv[r]);
+                    }
             }
         }
-        cp_async_wait_all(); // v gathers and early U_k fetches have landed
-        helper_bar();        // table built, staging area free
-        // ---- S5: non-zeros of block b+1 into the staging area
-        if (!hdr_warp && b + 1 < nblocks) issue_entries(b + 1);
         // ---- S6: the chain must have finished block b-1 before its table is read
         if (have_prev) done_wait();
+        else helper_bar();
         const bool write_back_first = have_prev && !prev_slow && slow; // an unstaged block reads global memory
         if (write_back_first) {
             for (int i = ht; i < Prev.n_occ; i += kHelperThreads) {
                 const int p = Prev.occ[i];
-                Uk[Prev.key[p]] = TuPrev[p];
+                Uk[Prev.key[p]] = (TwPrev[p] - Prev.Tv[p]) * inv_sigma;
             }
         }
         // ---- S7: complete the table: carried slots from the previous table, late fetches
@@ -442,8 +540,8 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                 for (int r = 0; r < 4; ++r) cc[r] = pp[r] < HTC ? B.carry[pp[r]] : kNoCarry;
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
-                    if (cc[r] != kNoCarry) Tu[pp[r]] = TuPrev[cc[r]];
-                    else if (!early_ok && pp[r] < HTC) Tu[pp[r]] = __ldcg(Uk + B.key[pp[r]]);
+                    if (cc[r] != kNoCarry) Tw[pp[r]] = TwPrev[cc[r]];
+                    else if (!early_ok && pp[r] < HTC) Tw[pp[r]] = fmaf(P.sigma, __ldcg(Uk + B.key[pp[r]]), B.Tv[pp[r]]);
                 }
             }
         }
@@ -453,26 +551,36 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
         }
         full_arrive(); // block b is ready (every helper's writes are ordered before its arrival)
         // ---- the previous block's results go back to global memory, off the chain's critical path
-        if (have_prev && !P.multi_epoch && ht < Prev.cnt) P.alpha[Prev.hdr[ht].coord] = Prev.hdr[ht].p1;
+        if (have_prev && !P.multi_epoch && ht < Prev.cnt) {
+            const float a_new = Prev.hdr[ht].p1;
+            if (!(fabsf(a_new) <= CUDART_MAX_NORMAL_F)) atomicOr(P.status, ST_NONFINITE_STEP);
+            P.alpha[Prev.hdr[ht].coord] = a_new;
+        }
         if (have_prev && !prev_slow && !write_back_first) {
             for (int i = ht; i < Prev.n_occ; i += kHelperThreads) {
                 const int p = Prev.occ[i];
-                Uk[Prev.key[p]] = TuPrev[p];
+                Uk[Prev.key[p]] = (TwPrev[p] - Prev.Tv[p]) * inv_sigma;
             }
         }
         helper_bar(); // the previous buffer may be rebuilt, and its global values are in place
     }
-    // ---- epilogue: the last block's results
+    // ---- epilogue: the last block's results and the hot ids
     {
         const int64_t b = nblocks - 1;
         Buf &L = sh.buf[b & 1];
+        const float *TwL = sh.W + HOT + (b & 1) * HTC;
         done_wait();
-        if (!P.multi_epoch && ht < L.cnt) P.alpha[L.hdr[ht].coord] = L.hdr[ht].p1;
+        if (!P.multi_epoch && ht < L.cnt) {
+            const float a_new = L.hdr[ht].p1;
+            if (!(fabsf(a_new) <= CUDART_MAX_NORMAL_F)) atomicOr(P.status, ST_NONFINITE_STEP);
+            P.alpha[L.hdr[ht].coord] = a_new;
+        }
         if (!L.slow)
             for (int i = ht; i < L.n_occ; i += kHelperThreads) {
                 const int p = L.occ[i];
-                Uk[L.key[p]] = sh.U[HOT + (b & 1) * HTC + p];
+                Uk[L.key[p]] = (TwL[p] - L.Tv[p]) * inv_sigma;
             }
+        for (int i = ht; i < hot_n; i += kHelperThreads) Uk[i] = (sh.W[i] - P.vbase[i]) * inv_sigma;
     }
 }
 
