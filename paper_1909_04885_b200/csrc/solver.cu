@@ -356,6 +356,7 @@ size_t smem_bytes(bool dense, int cap, int nslot)
 } // namespace
 
 cudaError_t launch_blocked_solver(Glm &g, const SolverParams &P);
+int blocked_solver_max_dense_dim();
 
 bool solver_supports_dense(int64_t dim, int max_smem_optin)
 {
@@ -391,14 +392,19 @@ cudaError_t launch_local_solver(Glm &g, int64_t H, float sigma_prime, int *varia
     const bool dense = g.fmt == CHICLE_FMT_DENSE_ROWMAJOR;
     const size_t budget = (size_t)g.max_smem_optin;
     int cap, nslot = 64; // a multiple of the producer warp count; each producer owns nslot / P slots
+    const char *force = getenv("CHICLE_FORCE_VARIANT"); // debugging aid: "ring" selects the unblocked solver
+    const bool ring = force && strcmp(force, "ring") == 0;
+    if (dense && g.dim <= blocked_solver_max_dense_dim() && !ring) {
+        *variant = 3;
+        return launch_blocked_solver(g, P);
+    }
     if (dense) {
         cap = (int)((g.dim + 31) / 32 * 32);
         while (nslot > 4 && smem_bytes(true, cap, nslot) > budget) nslot /= 2;
         if (smem_bytes(true, cap, nslot) > budget) return cudaErrorInvalidConfiguration;
         *variant = 0;
     } else {
-        const char *force = getenv("CHICLE_FORCE_VARIANT"); // debugging aid: "ring" selects the unblocked sparse solver
-        if (!(force && strcmp(force, "ring") == 0)) {
+        if (!ring) {
             *variant = 1;
             return launch_blocked_solver(g, P);
         }

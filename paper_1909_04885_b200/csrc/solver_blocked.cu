@@ -1,4 +1,4 @@
-// Local SCD solver for sparse coordinates (CSR rows / CSC columns): one CTA per partition, the visiting order
+// Local SCD solver for sparse coordinates (CSR rows / CSC columns) and for short dense rows: one CTA per partition, the visiting order
 // walked strictly in order (paper Sec. 2.1 worker structure with L = 1; Sec. 5.1: SCD local solver), with the
 // part of the local model that the next steps can touch held in shared memory.
 //
@@ -120,8 +120,8 @@ template <int CHUNKS> struct StepRaw {
     uint32_t s[CHUNKS];
     float x[CHUNKS];
 };
-template <int CHUNKS, int CAP>
-__device__ __forceinline__ void issue_step(StepRaw<CHUNKS> &r, int j, uint32_t hdr0, uint32_t pos0, uint32_t val0)
+template <int CHUNKS, int CAP, bool DENSE>
+__device__ __forceinline__ void issue_step(StepRaw<CHUNKS> &r, int j, uint32_t hdr0, uint32_t pos0, uint32_t val0, int lane)
 {
     const uint32_t hb = hdr0 + 48u * j;
     r.hi = lds_s32x4(hb);
@@ -129,7 +129,9 @@ __device__ __forceinline__ void issue_step(StepRaw<CHUNKS> &r, int j, uint32_t h
     const uint32_t pb = pos0 + (uint32_t)(2 * CAP) * j, xb = val0 + (uint32_t)(4 * CAP) * j;
 #pragma unroll
     for (int c = 0; c < CHUNKS; ++c) {
-        r.s[c] = lds_u16(pb + 64u * c); // always a valid shared address; the content counts only if active
+        // dense rows: entry e of a row is simply id e; otherwise the staged slot (always a valid shared address to
+        // read; the content counts only if the lane is active)
+        r.s[c] = DENSE ? (uint32_t)(lane + 32 * c) : lds_u16(pb + 64u * c);
         r.x[c] = lds_f32(xb + 128u * c);
     }
 }
@@ -149,7 +151,7 @@ __device__ __forceinline__ void finish_step(StepRegs<CHUNKS> &r, const StepRaw<C
     }
 }
 
-template <int LOSS, int HOT, int HTC, int CAP>
+template <int LOSS, bool DENSE, int HOT, int HTC, int CAP>
 __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const SolverParams P)
 {
     static_assert((HTC & (HTC - 1)) == 0 && HOT + 2 * HTC + 32 <= 65535 && CAP % 32 == 0 && CAP <= 252, "slot encoding");
@@ -200,10 +202,10 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                 const uint32_t val0 = smem_u32(&B.val[0][0]) + 4u * lane;
                 StepRegs<kChunks> cur;
                 StepRaw<kChunks> raw;
-                issue_step<kChunks, CAP>(raw, 0, hdr0, pos0, val0);
+                issue_step<kChunks, CAP, DENSE>(raw, 0, hdr0, pos0, val0, lane);
                 finish_step<kChunks>(cur, raw, wbase, dummy, lane);
                 for (int j = 0; j < cnt; ++j) {
-                    if (j + 1 < cnt) issue_step<kChunks, CAP>(raw, j + 1, hdr0, pos0, val0);
+                    if (j + 1 < cnt) issue_step<kChunks, CAP, DENSE>(raw, j + 1, hdr0, pos0, val0, lane);
                     SlotHdr h;
                     h.row_start = 0;
                     h.coord = cur.coord;
@@ -244,7 +246,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                     const int32_t *ix = P.indices + h.row_start;
                     const float *xv = P.values + h.row_start;
                     for (int e = lane; e < h.nnz; e += 32) {
-                        const int32_t i = ix[e];
+                        const int32_t i = DENSE ? e : ix[e];
                         const float ww = i < hot_n ? sh.W[i] : fmaf(sigma, Uk[i], P.vbase[i]);
                         acc = fmaf(xv[e], ww, acc);
                     }
@@ -257,7 +259,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                     }
                     if (delta != 0.0f)
                         for (int e = lane; e < h.nnz; e += 32) {
-                            const int32_t i = ix[e];
+                            const int32_t i = DENSE ? e : ix[e];
                             if (i < hot_n) sh.W[i] = fmaf(sigma * delta, xv[e], sh.W[i]);
                             else Uk[i] = fmaf(delta, xv[e], Uk[i]);
                         }
@@ -293,8 +295,13 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
     auto issue_fields = [&](int32_t c) -> Fields {
         Fields f{c, 0, 0, 0.f, 0.f, 0.f};
         if (c >= 0) {
-            f.rs = P.indptr[c];
-            f.re = P.indptr[c + 1];
+            if (DENSE) {
+                f.rs = (int64_t)c * P.dim;
+                f.re = f.rs + P.dim;
+            } else {
+                f.rs = P.indptr[c];
+                f.re = P.indptr[c + 1];
+            }
             f.s = P.sqnorm[c];
             f.al = __ldcg(P.alpha + c);
             if (LOSS != CHICLE_LOSS_RIDGE_PRIMAL) f.y = P.labels[c];
@@ -345,14 +352,14 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
             first = f.rs & ~(int64_t)3;
             bytes = (uint32_t)(((f.re - first) + 3) & ~(int64_t)3) * 4u;
         }
-        uint32_t total = 2u * bytes;
+        uint32_t total = DENSE ? bytes : 2u * bytes;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
         const uint32_t bar = smem_u32(&st.bar);
         if (lane == 0) mbar_arrive_expect_tx(bar, total);
         __syncwarp();
         if (bytes) {
-            bulk_g2s(smem_u32(&st.idx[lane][0]), P.indices + first, bytes, bar);
+            if (!DENSE) bulk_g2s(smem_u32(&st.idx[lane][0]), P.indices + first, bytes, bar);
             bulk_g2s(smem_u32(&st.val[lane][0]), P.values + first, bytes, bar);
         }
     };
@@ -418,10 +425,12 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                     const int e = e0 + lane;
                     bool cold = false;
                     if (e < nnz) {
-                        const int32_t idx = st.idx[j][sft + e];
                         B.val[j][e] = st.val[j][sft + e];
-                        if (HOT > 0 && idx < HOT) B.pos[j][e] = (uint16_t)idx;
-                        else cold = true;
+                        if (!DENSE) {
+                            const int32_t idx = st.idx[j][sft + e];
+                            if (HOT > 0 && idx < HOT) B.pos[j][e] = (uint16_t)idx;
+                            else cold = true;
+                        }
                     }
                     const uint32_t m = __ballot_sync(0xffffffffu, cold);
                     if (m) {
@@ -584,11 +593,11 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
     }
 }
 
-template <int LOSS, int HOT, int HTC, int CAP> cudaError_t launch_one(Glm &g, const SolverParams &P)
+template <int LOSS, bool DENSE, int HOT, int HTC, int CAP> cudaError_t launch_one(Glm &g, const SolverParams &P)
 {
     using Shared = SharedB<HOT, HTC, CAP>;
     static_assert(sizeof(Shared) <= 227 * 1024, "shared memory budget");
-    auto kern = k_local_scd_blocked<LOSS, HOT, HTC, CAP>;
+    auto kern = k_local_scd_blocked<LOSS, DENSE, HOT, HTC, CAP>;
     const size_t smem = sizeof(Shared);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -600,16 +609,20 @@ template <int LOSS, int HOT, int HTC, int CAP> cudaError_t launch_one(Glm &g, co
 constexpr int kHotA = 24576, kHtcA = 1024, kCapA = 96;
 // flat ids: no direct array, everything through the table
 constexpr int kHotB = 0, kHtcB = 4096, kCapB = 128;
+// short dense rows: entry e of every row is id e, all of w_local is "hot", no table
+constexpr int kHotD = 128, kHtcD = 32, kCapD = 128;
 
 template <int LOSS> cudaError_t launch_loss(Glm &g, const SolverParams &P)
 {
-    if (g.hot_variant) return launch_one<LOSS, kHotA, kHtcA, kCapA>(g, P);
-    return launch_one<LOSS, kHotB, kHtcB, kCapB>(g, P);
+    if (g.fmt == CHICLE_FMT_DENSE_ROWMAJOR) return launch_one<LOSS, true, kHotD, kHtcD, kCapD>(g, P);
+    if (g.hot_variant) return launch_one<LOSS, false, kHotA, kHtcA, kCapA>(g, P);
+    return launch_one<LOSS, false, kHotB, kHtcB, kCapB>(g, P);
 }
 
 } // namespace
 
 int blocked_solver_hot_ids() { return kHotA; }
+int blocked_solver_max_dense_dim() { return kCapD; }
 
 cudaError_t launch_blocked_solver(Glm &g, const SolverParams &P)
 {
