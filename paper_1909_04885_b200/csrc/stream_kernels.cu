@@ -90,7 +90,7 @@ k_reduce_updates(float *__restrict__ v, float *__restrict__ U, int K, int64_t di
         } else {
             acc[0] = v[i];
         }
-#pragma unroll 8
+#pragma unroll 16
         for (int k = 0; k < K; ++k) {
             if (VEC == 4) {
                 float4 *p = reinterpret_cast<float4 *>(U + (size_t)k * dim) + i;
@@ -125,12 +125,46 @@ __global__ void k_resid(const float *__restrict__ v, const float *__restrict__ y
 }
 
 // ---------------------------------------------------------------------------------------- duality gap (a6)
-// One pass over the coordinate-major matrix: a warp per coordinate computes its dot product with the shared
-// vector in fp64 and the coordinate's term; lane 0 of every warp keeps running fp64 sums over the coordinates it
-// was assigned (a fixed assignment), the block adds its warps in order and writes 4 partial sums; a second kernel
-// adds the blocks in order. Partials: dual losses {sum loss, sum gap term, |v|^2 slice, 0};
+// One streaming pass over the coordinate-major matrix. Sparse: a warp takes four consecutive coordinates at a time
+// and issues all their index/value loads (then all gathers from the shared vector) before reducing anything, so
+// that enough bytes are in flight to cover the memory latency; dot products and sums are fp64. Short dense rows: a
+// thread per row with 128-bit loads. Lanes keep running fp64 sums over the coordinates they were assigned (a fixed
+// assignment), the block adds its lanes and warps in a fixed order and writes 4 partial sums; a second kernel adds
+// the blocks in a fixed order. Partials: dual losses {sum loss, sum gap term, |v|^2 slice, 0};
 // ridge {sum (c_j . r)^2, sum w_j^2, sum r^2 slice, sum r*y slice} with r = v - y.
 __device__ __forceinline__ double xlogx(double x) { return x > 0.0 ? x * log(x) : 0.0; }
+
+// adds coordinate c's contribution, given its dot product with the shared vector (with v - y for ridge)
+template <int LOSS>
+__device__ __forceinline__ void gap_term(double dot, float label, float state, double lam_n, double &s0, double &s1)
+{
+    if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+        const double w = (double)state;
+        s0 += dot * dot;
+        s1 += w * w;
+    } else {
+        const double y = (double)label;
+        const double mu = y * dot / lam_n;
+        double a = y * (double)state;
+        a = a < 0.0 ? 0.0 : (a > 1.0 ? 1.0 : a);
+        double l, conj;
+        if (LOSS == CHICLE_LOSS_HINGE_DUAL) {
+            l = 1.0 - mu > 0.0 ? 1.0 - mu : 0.0;
+            conj = -a;
+        } else {
+            l = mu < 0.0 ? -mu + log1p(exp(mu)) : log1p(exp(-mu));
+            conj = xlogx(a) + xlogx(1.0 - a);
+        }
+        s0 += l;
+        s1 += l + conj + a * mu;
+    }
+}
+
+#ifndef CHICLE_GAP_ROWS
+#define CHICLE_GAP_ROWS 4
+#endif
+constexpr int kGapRows = CHICLE_GAP_ROWS;   // coordinates a warp has in flight
+constexpr int kGapChunks = 2; // 32-entry chunks per coordinate held in registers (longer ones loop)
 
 template <int LOSS>
 __global__ void __launch_bounds__(kThreads)
@@ -139,48 +173,107 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
                const float *__restrict__ vec /* the shared vector */, const float *__restrict__ v,
                int64_t n_coord, int64_t dim, double lam_n, double *__restrict__ partials)
 {
-    __shared__ double sh[kWarpsPerBlock][4];
+    __shared__ double sh[kThreads][2];
+    __shared__ double sh2[kWarpsPerBlock][2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t nw = (int64_t)gridDim.x * kWarpsPerBlock;
+    const int64_t gw = (int64_t)blockIdx.x * kWarpsPerBlock + warp;
     double s0 = 0.0, s1 = 0.0;
-    for (int64_t c = (int64_t)blockIdx.x * kWarpsPerBlock + warp; c < n_coord; c += nw) {
-        double dot = 0.0;
-        if (indptr) {
-            const int64_t b = indptr[c], e = indptr[c + 1];
-            if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
-                for (int64_t q = b + lane; q < e; q += 32) {
-                    const int32_t r = indices[q];
-                    dot = fma((double)values[q], (double)vec[r] - (double)labels[r], dot);
-                }
-            } else {
-                for (int64_t q = b + lane; q < e; q += 32) dot = fma((double)values[q], (double)vec[indices[q]], dot);
+    if (indptr) {
+        const int64_t ngroups = (n_coord + kGapRows - 1) / kGapRows;
+        // the row pointers and per-coordinate scalars of a group are fetched one iteration ahead
+        auto fetch_ip = [&](int64_t g) -> int64_t {
+            if (g >= ngroups || lane > kGapRows) return 0;
+            const int64_t c = g * kGapRows + lane;
+            return indptr[c < n_coord ? c : n_coord];
+        };
+        auto fetch_scalars = [&](int64_t g, float &lab, float &sta) {
+            lab = 0.0f;
+            sta = 0.0f;
+            const int64_t c = g * kGapRows + lane;
+            if (g < ngroups && lane < kGapRows && c < n_coord) {
+                sta = state[c];
+                if (LOSS != CHICLE_LOSS_RIDGE_PRIMAL) lab = labels[c];
             }
-        } else {
-            const float *row = values + c * dim;
-            for (int64_t j = lane; j < dim; j += 32) dot = fma((double)row[j], (double)vec[j], dot);
+        };
+        int64_t ip_next = fetch_ip(gw);
+        float lab_next, sta_next;
+        fetch_scalars(gw, lab_next, sta_next);
+        for (int64_t g = gw; g < ngroups; g += nw) {
+            const int64_t c0 = g * kGapRows;
+            const int64_t ip = ip_next;
+            const float my_label = lab_next, my_state = sta_next;
+            ip_next = fetch_ip(g + nw);
+            fetch_scalars(g + nw, lab_next, sta_next);
+            const bool owner = lane < kGapRows && c0 + lane < n_coord;
+            int64_t rs[kGapRows], re[kGapRows];
+#pragma unroll
+            for (int r = 0; r < kGapRows; ++r) {
+                rs[r] = __shfl_sync(0xffffffffu, ip, r);
+                re[r] = __shfl_sync(0xffffffffu, ip, r + 1);
+            }
+            int32_t ix[kGapRows][kGapChunks];
+            float xv[kGapRows][kGapChunks];
+#pragma unroll
+            for (int r = 0; r < kGapRows; ++r)
+#pragma unroll
+                for (int ch = 0; ch < kGapChunks; ++ch) {
+                    const int64_t e = rs[r] + lane + 32 * ch;
+                    ix[r][ch] = -1;
+                    xv[r][ch] = 0.0f;
+                    if (e < re[r]) {
+                        ix[r][ch] = indices[e];
+                        xv[r][ch] = values[e];
+                    }
+                }
+            double dot[kGapRows];
+#pragma unroll
+            for (int r = 0; r < kGapRows; ++r) {
+                dot[r] = 0.0;
+#pragma unroll
+                for (int ch = 0; ch < kGapChunks; ++ch)
+                    if (ix[r][ch] >= 0) {
+                        double t = (double)vec[ix[r][ch]];
+                        if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) t -= (double)labels[ix[r][ch]];
+                        dot[r] = fma((double)xv[r][ch], t, dot[r]);
+                    }
+                for (int64_t e = rs[r] + 32 * kGapChunks + lane; e < re[r]; e += 32) { // the rest of a long coordinate
+                    const int32_t i = indices[e];
+                    double t = (double)vec[i];
+                    if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) t -= (double)labels[i];
+                    dot[r] = fma((double)values[e], t, dot[r]);
+                }
+            }
+            double mine = 0.0;
+#pragma unroll
+            for (int r = 0; r < kGapRows; ++r) {
+                const double d = warp_sum_d(dot[r]);
+                if (lane == r) mine = d;
+            }
+            if (owner) gap_term<LOSS>(mine, my_label, my_state, lam_n, s0, s1);
         }
-        dot = warp_sum_d(dot);
-        if (lane == 0) {
-            if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
-                const double w = (double)state[c];
-                s0 += dot * dot;
-                s1 += w * w;
-            } else {
-                const double y = (double)labels[c];
-                const double mu = y * dot / lam_n;
-                double a = y * (double)state[c];
-                a = a < 0.0 ? 0.0 : (a > 1.0 ? 1.0 : a);
-                double l, conj;
-                if (LOSS == CHICLE_LOSS_HINGE_DUAL) {
-                    l = 1.0 - mu > 0.0 ? 1.0 - mu : 0.0;
-                    conj = -a;
-                } else {
-                    l = mu < 0.0 ? -mu + log1p(exp(mu)) : log1p(exp(-mu));
-                    conj = xlogx(a) + xlogx(1.0 - a);
-                }
-                s0 += l;
-                s1 += l + conj + a * mu;
+    } else if (dim <= 64 && (dim & 3) == 0) {
+        // short dense rows: a thread per row, 128-bit loads; a warp's 32 rows are contiguous in memory
+        const int64_t stride = (int64_t)gridDim.x * kThreads;
+        for (int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x; c < n_coord; c += stride) {
+            const float4 *row = reinterpret_cast<const float4 *>(values + c * dim);
+            double dot = 0.0;
+            for (int j4 = 0; j4 < (int)(dim >> 2); ++j4) {
+                const float4 x = row[j4];
+                dot = fma((double)x.x, (double)vec[4 * j4], dot);
+                dot = fma((double)x.y, (double)vec[4 * j4 + 1], dot);
+                dot = fma((double)x.z, (double)vec[4 * j4 + 2], dot);
+                dot = fma((double)x.w, (double)vec[4 * j4 + 3], dot);
             }
+            gap_term<LOSS>(dot, labels[c], state[c], lam_n, s0, s1);
+        }
+    } else {
+        for (int64_t c = gw; c < n_coord; c += nw) {
+            const float *row = values + c * dim;
+            double dot = 0.0;
+            for (int64_t j = lane; j < dim; j += 32) dot = fma((double)row[j], (double)vec[j], dot);
+            dot = warp_sum_d(dot);
+            if (lane == 0) gap_term<LOSS>(dot, labels[c], state[c], lam_n, s0, s1);
         }
     }
     // slice of the shared vector owned by this block
@@ -203,14 +296,29 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
         s2 = warp_sum_d(s2);
         s3 = warp_sum_d(s3);
     }
+    // fixed-order combination: threads in index order for the per-coordinate sums, warps in order for the slices
+    sh[threadIdx.x][0] = s0;
+    sh[threadIdx.x][1] = s1;
     if (lane == 0) {
-        sh[warp][0] = s0; sh[warp][1] = s1; sh[warp][2] = s2; sh[warp][3] = s3;
+        sh2[warp][0] = s2;
+        sh2[warp][1] = s3;
     }
     __syncthreads();
-    if (threadIdx.x < 4) {
-        double t = 0.0;
-        for (int w = 0; w < kWarpsPerBlock; ++w) t += sh[w][threadIdx.x];
-        partials[(size_t)blockIdx.x * 4 + threadIdx.x] = t;
+    if (threadIdx.x < 2) {
+        // pairwise tree over the 256 threads, fixed shape
+        double t[kThreads / 32];
+        for (int w = 0; w < kThreads / 32; ++w) {
+            double a = 0.0;
+            for (int l = 0; l < 32; ++l) a += sh[w * 32 + l][threadIdx.x];
+            t[w] = a;
+        }
+        double tot = 0.0;
+        for (int w = 0; w < kThreads / 32; ++w) tot += t[w];
+        partials[(size_t)blockIdx.x * 4 + threadIdx.x] = tot;
+    } else if (threadIdx.x < 4) {
+        double tot = 0.0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) tot += sh2[w][threadIdx.x - 2];
+        partials[(size_t)blockIdx.x * 4 + threadIdx.x] = tot;
     }
 }
 
@@ -218,11 +326,18 @@ template <int LOSS>
 __global__ void k_gap_final(const double *__restrict__ partials, int nblocks, double n, double lambda,
                             double *__restrict__ out)
 {
+    // 4 warps, one per partial sum: lane l adds blocks l, l+32, ... in order, then the 32 lanes are added in order
+    __shared__ double lanes[4][32];
     __shared__ double tot[4];
+    const int q = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    double t = 0.0;
+    for (int b = lane; b < nblocks; b += 32) t += partials[(size_t)b * 4 + q];
+    lanes[q][lane] = t;
+    __syncthreads();
     if (threadIdx.x < 4) {
-        double t = 0.0;
-        for (int b = 0; b < nblocks; ++b) t += partials[(size_t)b * 4 + threadIdx.x];
-        tot[threadIdx.x] = t;
+        double a = 0.0;
+        for (int l = 0; l < 32; ++l) a += lanes[threadIdx.x][l];
+        tot[threadIdx.x] = a;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -291,9 +406,10 @@ cudaError_t launch_reduce(Glm &g)
     float *resid = g.loss == CHICLE_LOSS_RIDGE_PRIMAL ? g.resid : nullptr;
     if ((g.dim & 3) == 0) {
         const int64_t nvec = g.dim / 4;
-        unsigned grid = blocks_for(nvec, kThreads);
+        const int threads = nvec >= (int64_t)g.sm_count * 2 * kThreads ? kThreads : 64; // small vectors: more, smaller blocks
+        unsigned grid = blocks_for(nvec, threads);
         if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
-        k_reduce_updates<4><<<grid, kThreads, 0, g.stream>>>(g.v, g.U, g.K, g.dim, y, resid);
+        k_reduce_updates<4><<<grid, threads, 0, g.stream>>>(g.v, g.U, g.K, g.dim, y, resid);
     } else {
         unsigned grid = blocks_for(g.dim, kThreads);
         if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
@@ -318,18 +434,18 @@ cudaError_t launch_gap(Glm &g)
     case CHICLE_LOSS_HINGE_DUAL:
         k_gap_partials<CHICLE_LOSS_HINGE_DUAL><<<nb, kThreads, 0, g.stream>>>(
             g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord, g.dim, lam_n, g.gap_partials);
-        k_gap_final<CHICLE_LOSS_HINGE_DUAL><<<1, 32, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda, g.gap_out);
+        k_gap_final<CHICLE_LOSS_HINGE_DUAL><<<1, 128, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda, g.gap_out);
         break;
     case CHICLE_LOSS_LOGISTIC_DUAL:
         k_gap_partials<CHICLE_LOSS_LOGISTIC_DUAL><<<nb, kThreads, 0, g.stream>>>(
             g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord, g.dim, lam_n, g.gap_partials);
-        k_gap_final<CHICLE_LOSS_LOGISTIC_DUAL><<<1, 32, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda,
+        k_gap_final<CHICLE_LOSS_LOGISTIC_DUAL><<<1, 128, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda,
                                                                         g.gap_out);
         break;
     default:
         k_gap_partials<CHICLE_LOSS_RIDGE_PRIMAL><<<nb, kThreads, 0, g.stream>>>(
             g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord, g.dim, lam_n, g.gap_partials);
-        k_gap_final<CHICLE_LOSS_RIDGE_PRIMAL><<<1, 32, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda,
+        k_gap_final<CHICLE_LOSS_RIDGE_PRIMAL><<<1, 128, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda,
                                                                        g.gap_out);
         break;
     }
