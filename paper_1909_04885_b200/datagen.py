@@ -71,8 +71,11 @@ class Workload:
         return cur
 
 
+_DEVICE = "cpu"   # where make() draws; "cuda" makes the two largest configurations practical (other random stream)
+
+
 def _gen(seed: int) -> torch.Generator:
-    g = torch.Generator(device="cpu")
+    g = torch.Generator(device=_DEVICE)
     g.manual_seed(int(seed))
     return g
 
@@ -167,7 +170,7 @@ def hinge_dense(scale: int = 1, seed: int = 0) -> Workload:
     w = torch.randn(d, generator=g, dtype=torch.float64)
     y = _sign_pm1(X.double() @ w + 0.1 * torch.randn(n, generator=g, dtype=torch.float64)).float()
     K = 4
-    return Workload("hinge_dense", "hinge", "dense", n, d, X.reshape(-1).numpy(), y.numpy(), 1.0 / n, 10,
+    return Workload("hinge_dense", "hinge", "dense", n, d, X.reshape(-1).cpu().numpy(), y.cpu().numpy(), 1.0 / n, 10,
                     [Phase(0, K, seed, float(K))])
 
 
@@ -185,8 +188,8 @@ def hinge_csr(scale: int = 1, seed: int = 0, mean_nnz: float = 50.0, zipf_s: flo
     y = _sign_pm1(score)
     flip = torch.rand(n, generator=g, dtype=torch.float64) < 0.05
     y = torch.where(flip, -y, y).float()
-    return Workload(name, "hinge", "csr", n, d, vals.numpy(), y.numpy(), lam * scale, rounds,
-                    [Phase(0, K, seed, float(K))], indptr.numpy(), idx.numpy(),
+    return Workload(name, "hinge", "csr", n, d, vals.cpu().numpy(), y.cpu().numpy(), lam * scale, rounds,
+                    [Phase(0, K, seed, float(K))], indptr.cpu().numpy(), idx.cpu().numpy(),
                     meta={"lambda_note": "lambda*n kept constant when scaled"})
 
 
@@ -201,7 +204,7 @@ def logistic_dense(scale: int = 1, seed: int = 0) -> Workload:
     p = torch.sigmoid(X.double() @ w)
     y = torch.where(torch.rand(n, generator=g, dtype=torch.float64) < p, 1.0, -1.0).float()
     K = 32
-    return Workload("logistic_dense", "logistic", "dense", n, d, X.reshape(-1).numpy(), y.numpy(), 1e-6 * scale, 20,
+    return Workload("logistic_dense", "logistic", "dense", n, d, X.reshape(-1).cpu().numpy(), y.cpu().numpy(), 1e-6 * scale, 20,
                     [Phase(0, K, seed, float(K))], meta={"lambda_note": "lambda*n kept at 11 when scaled"})
 
 
@@ -219,8 +222,8 @@ def hinge_hashed(scale: int = 1, seed: int = 0) -> Workload:
     head = score[: min(n, 1_000_000)]
     thr = torch.quantile(head[: min(head.numel(), 1 << 24)], 0.75)
     y = torch.where(score > thr, 1.0, -1.0).float()
-    return Workload("hinge_hashed", "hinge", "csr", n, d, vals.numpy(), y.numpy(), 1e-7 * scale, 30,
-                    [Phase(0, 64, seed, 64.0), Phase(10, 16, seed + 1, 16.0)], indptr.numpy(), idx.numpy(),
+    return Workload("hinge_hashed", "hinge", "csr", n, d, vals.cpu().numpy(), y.cpu().numpy(), 1e-7 * scale, 30,
+                    [Phase(0, 64, seed, 64.0), Phase(10, 16, seed + 1, 16.0)], indptr.cpu().numpy(), idx.cpu().numpy(),
                     meta={"lambda_note": "lambda*n kept at 4.5 when scaled"})
 
 
@@ -241,8 +244,8 @@ def ridge_csc(scale: int = 1, seed: int = 0, mean_nnz: float = 3700.0) -> Worklo
     colptr = torch.zeros(d + 1, dtype=torch.int64)
     colptr[1:] = torch.cumsum(col_counts, 0)
     K = 128
-    return Workload("ridge_csc", "ridge", "csc", n, d, vals[order].numpy(), y.float().numpy(), 1e-4 * scale, 15,
-                    [Phase(0, K, seed, float(K))], colptr.numpy(), rows[order].to(torch.int32).numpy())
+    return Workload("ridge_csc", "ridge", "csc", n, d, vals[order].cpu().numpy(), y.float().cpu().numpy(), 1e-4 * scale, 15,
+                    [Phase(0, K, seed, float(K))], colptr.cpu().numpy(), rows[order].to(torch.int32).cpu().numpy())
 
 
 CONFIGS = {
@@ -254,5 +257,14 @@ CONFIGS = {
 }
 
 
-def make(name: str, scale: int = 1, seed: int = 0) -> Workload:
-    return CONFIGS[name](scale=scale, seed=seed)
+def make(name: str, scale: int = 1, seed: int = 0, device: str = "cpu") -> Workload:
+    """Draws a workload. ``device="cuda"`` draws with torch on the GPU (needed in practice for the two largest
+    configurations at full size; the random stream differs from the CPU one) and returns host arrays all the same."""
+    global _DEVICE
+    prev = _DEVICE
+    _DEVICE = device
+    try:
+        with torch.device(device):
+            return CONFIGS[name](scale=scale, seed=seed)
+    finally:
+        _DEVICE = prev

@@ -1,0 +1,36 @@
+"""The two largest configurations at full size (45 M x 1 M hashed CSR with the K = 64 -> 16 repartition; ridge on a
+350 k x 16 M CSC matrix), element by element against the oracle for a few rounds. Takes several minutes and about
+60 GB of host memory, so it only runs when CHICLE_FULL_SIZE=1; inputs are drawn on the GPU (datagen device="cuda")."""
+import os
+import time
+
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+full = pytest.mark.skipif(os.environ.get("CHICLE_FULL_SIZE") != "1", reason="set CHICLE_FULL_SIZE=1 to run")
+
+
+@full
+def test_config4_full_size_with_repartition():
+    from paper_1909_04885_b200 import datagen
+    from paper_1909_04885_b200.datagen import Phase
+    from parity_util import run_parity
+    t0 = time.time()
+    w = datagen.make("hinge_hashed", 1, device="cuda")
+    print("config 4 drawn in %.0f s: n=%d d=%d nnz=%d" % (time.time() - t0, w.n_rows, w.n_cols, w.nnz))
+    seed = w.phases[0].seed
+    w.phases = [Phase(0, 64, seed, 64.0), Phase(2, 16, seed + 1, 16.0)]
+    worst = run_parity(w, rounds=4)
+    print("config 4 worst relative errors", worst)
+
+
+@full
+def test_config5_full_size():
+    from paper_1909_04885_b200 import datagen
+    from parity_util import run_parity
+    t0 = time.time()
+    w = datagen.make("ridge_csc", 1, device="cuda")
+    print("config 5 drawn in %.0f s: n=%d d=%d nnz=%d" % (time.time() - t0, w.n_rows, w.n_cols, w.nnz))
+    worst = run_parity(w, rounds=3)
+    print("config 5 worst relative errors", worst)
