@@ -243,10 +243,10 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
         if (!ok2) return bail(CHICLE_ERR_OOM, "device allocation failed (id ranking)");
         e = cudaMemsetAsync(counts, 0, (size_t)dim * 4, s);
         if (e == cudaSuccess) e = cudaMemsetAsync(mass, 0, 32, s);
-        if (e == cudaSuccess) e = launch_frequency_remap(*h, counts, keys, vals, hist, sums, blocked_solver_hot_ids(), mass);
+        if (e == cudaSuccess) e = launch_frequency_remap(*h, counts, keys, vals, hist, sums, blocked_solver_hot_ids(), blocked_solver_short_cap(), mass);
         if (e == cudaSuccess && ridge) e = launch_gather_f32(*h, h->labels, h->old_of_new, dim, labels_new);
-        unsigned long long host_mass = 0;
-        if (e == cudaSuccess) e = cudaMemcpyAsync(&host_mass, mass, 8, cudaMemcpyDeviceToHost, s);
+        unsigned long long host_mass2[2] = {0, 0};
+        if (e == cudaSuccess) e = cudaMemcpyAsync(host_mass2, mass, 16, cudaMemcpyDeviceToHost, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
         if (e != cudaSuccess) return bail_cuda(e, "id ranking kernels");
         if (ridge) {
@@ -255,10 +255,13 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
         }
         dev_free(h, counts); dev_free(h, keys[0]); dev_free(h, keys[1]); dev_free(h, vals[0]); dev_free(h, vals[1]);
         dev_free(h, hist); dev_free(h, sums); dev_free(h, mass);
-        h->hot_variant = h->nnz > 0 && (double)host_mass >= 0.5 * (double)h->nnz ? 1 : 0;
+        h->hot_variant = h->nnz > 0 && (double)host_mass2[0] >= 0.5 * (double)h->nnz ? 1 : 0;
+        // more than 1 % of the coordinates would not fit the short staging rows: take the variant with longer rows
+        if (h->hot_variant && (double)host_mass2[1] > 0.01 * (double)h->n_coord) h->hot_variant = 2;
         const char *force = getenv("CHICLE_FORCE_VARIANT"); // debugging aid
         if (force && strcmp(force, "flat") == 0) h->hot_variant = 0;
         if (force && strcmp(force, "hot") == 0) h->hot_variant = 1;
+        if (force && strcmp(force, "hot128") == 0) h->hot_variant = 2;
     }
     e = launch_sqnorm(*h);
     if (e == cudaSuccess) e = launch_refresh_resid(*h);

@@ -78,7 +78,8 @@ struct Glm {
     int32_t *new_of_old = nullptr; // dim; nullptr when ids are not remapped (dense)
     int32_t *old_of_new = nullptr; // dim
     float *perm_tmp = nullptr;     // dim, staging for translating v at the boundary
-    int hot_variant = 0;           // 1: most non-zeros fall on the first ids, the solver keeps those in a direct array
+    int hot_variant = 0;           // 1 / 2: most non-zeros fall on the first ids, the solver keeps those in a direct
+                                   // array (2: with room for coordinates of up to 128 entries); 0: flat ids
 
     // partition
     int32_t K = 0;
@@ -118,8 +119,9 @@ cudaError_t launch_gap(Glm &g);                                           // fil
 cudaError_t launch_shared_vector(Glm &g);                                 // v = X^T alpha (or X w) from scratch
 cudaError_t launch_refresh_resid(Glm &g);                                 // ridge: resid = v - y
 cudaError_t launch_frequency_remap(Glm &g, uint32_t *counts, uint64_t *keys[2], int32_t *vals[2], uint32_t *hist,
-                                   uint32_t *scan_sums, int64_t hot_ids, unsigned long long *mass);
+                                   uint32_t *scan_sums, int64_t hot_ids, int32_t long_len, unsigned long long *mass);
 cudaError_t launch_gather_f32(Glm &g, const float *src, const int32_t *map, int64_t n, float *dst); // dst[i] = src[map[i]]
 int blocked_solver_hot_ids();
+int blocked_solver_short_cap();
 
 } // namespace chicle

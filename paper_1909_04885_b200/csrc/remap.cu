@@ -55,6 +55,18 @@ __global__ void k_mass_of_first(const uint32_t *__restrict__ counts, const int32
     if ((threadIdx.x & 31) == 0 && s) atomicAdd(out, s);
 }
 
+// out[1] += number of coordinates with more than `long_len` entries
+__global__ void k_count_long(const int64_t *__restrict__ indptr, int64_t n_coord, int32_t long_len,
+                             unsigned long long *__restrict__ out)
+{
+    unsigned long long s = 0;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < n_coord; c += (int64_t)gridDim.x * blockDim.x)
+        s += (indptr[c + 1] - indptr[c]) > long_len ? 1u : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if ((threadIdx.x & 31) == 0 && s) atomicAdd(out + 1, s);
+}
+
 // dst[i] = src[map[i]]
 __global__ void k_gather_f32(const float *__restrict__ src, const int32_t *__restrict__ map, int64_t n, float *__restrict__ dst)
 {
@@ -64,9 +76,10 @@ __global__ void k_gather_f32(const float *__restrict__ src, const int32_t *__res
 
 } // namespace
 
-// counts: dim zeroed uint32; keys/vals: two arrays of dim each; mass: one zeroed 64-bit word.
+// counts: dim zeroed uint32; keys/vals: two arrays of dim each; mass: two zeroed 64-bit words (non-zeros on the first
+// hot_ids ids; coordinates longer than long_len).
 cudaError_t launch_frequency_remap(Glm &g, uint32_t *counts, uint64_t *keys[2], int32_t *vals[2], uint32_t *hist,
-                                   uint32_t *scan_sums, int64_t hot_ids, unsigned long long *mass)
+                                   uint32_t *scan_sums, int64_t hot_ids, int32_t long_len, unsigned long long *mass)
 {
     const int64_t dim = g.dim;
     const unsigned wide = (unsigned)g.sm_count * 8;
@@ -83,6 +96,7 @@ cudaError_t launch_frequency_remap(Glm &g, uint32_t *counts, uint64_t *keys[2], 
     k_relabel<<<wide, kT, 0, g.stream>>>(g.indices, g.nnz, g.new_of_old);
     const int64_t first = hot_ids < dim ? hot_ids : dim;
     k_mass_of_first<<<blocks_for(first), kT, 0, g.stream>>>(counts, g.old_of_new, first, mass);
+    k_count_long<<<wide, kT, 0, g.stream>>>(g.indptr, g.n_coord, long_len, mass);
     return cudaGetLastError();
 }
 

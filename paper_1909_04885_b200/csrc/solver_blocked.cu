@@ -387,7 +387,16 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
         float *TwPrev = sh.W + HOT + (q ^ 1) * HTC; // the previous block's
         const bool have_prev = b > 0;
         // ---- S0: reset this buffer's table (its previous block was written back in the last iteration)
-        for (int p = ht; p < HTC; p += kHelperThreads) B.key[p] = -1;
+        // (the helpers' loops use explicit shared addresses too: generic accesses cost them several times more)
+        const uint32_t a_key = smem_u32(&B.key[0]), a_occ = smem_u32(&B.occ[0]), a_carry = smem_u32(&B.carry[0]);
+        const uint32_t a_tv = smem_u32(&B.Tv[0]), a_tw = smem_u32(Tw), a_twp = smem_u32(TwPrev);
+        const uint32_t a_keyp = smem_u32(&Prev.key[0]);
+        const uint32_t a_bval = smem_u32(&B.val[0][0]), a_bpos = smem_u32(&B.pos[0][0]);
+        const uint32_t a_sidx = smem_u32(&st.idx[0][0]), a_sval = smem_u32(&st.val[0][0]);
+        const uint32_t a_cold = smem_u32(&st.cold[0]), a_ncold = smem_u32(&st.n_cold), a_nocc = smem_u32(&B.n_occ);
+        const uint32_t a_hdrq = smem_u32(&st.hdr[q][0]), a_shiftq = smem_u32(&st.shift[q][0]);
+        constexpr uint32_t kStageRow = (CAP + 4) * 4; // bytes per staged coordinate
+        for (int p = ht; p < HTC; p += kHelperThreads) sts_s32(a_key + 4u * p, -1);
         if (ht == 0) {
             B.n_occ = 0;
             st.n_cold = 0;
@@ -419,16 +428,17 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
             // ---- S3a: classify. An entry warp takes whole coordinates, lanes over the non-zeros: copy the value,
             //      give hot ids their index, collect cold ones in a list.
             for (int j = ew; j < cnt; j += kEntryWarps) {
-                const int nnz = st.hdr[q][j].nnz;
-                const int sft = st.shift[q][j];
+                const int nnz = lds_s32(a_hdrq + 48u * j + 12u);
+                const int sft = lds_s32(a_shiftq + 4u * j);
+                const uint32_t srow = kStageRow * j + 4u * sft;
                 for (int e0 = 0; e0 < nnz; e0 += 32) {
                     const int e = e0 + lane;
                     bool cold = false;
                     if (e < nnz) {
-                        B.val[j][e] = st.val[j][sft + e];
+                        sts_f32(a_bval + (uint32_t)(4 * CAP) * j + 4u * e, lds_f32(a_sval + srow + 4u * e));
                         if (!DENSE) {
-                            const int32_t idx = st.idx[j][sft + e];
-                            if (HOT > 0 && idx < HOT) B.pos[j][e] = (uint16_t)idx;
+                            const int32_t idx = lds_s32(a_sidx + srow + 4u * e);
+                            if (HOT > 0 && idx < HOT) sts_u16(a_bpos + (uint32_t)(2 * CAP) * j + 2u * e, (uint32_t)idx);
                             else cold = true;
                         }
                     }
@@ -436,9 +446,9 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                     if (m) {
                         const int leader = __ffs(m) - 1;
                         int base = 0;
-                        if (lane == leader) base = atomicAdd(&st.n_cold, __popc(m));
+                        if (lane == leader) base = atoms_add(a_ncold, __popc(m));
                         base = __shfl_sync(0xffffffffu, base, leader);
-                        if (cold) st.cold[base + __popc(m & lt_mask)] = (uint16_t)((j << 8) | e);
+                        if (cold) sts_u16(a_cold + 2u * (base + __popc(m & lt_mask)), (uint32_t)((j << 8) | e));
                     }
                 }
             }
@@ -446,37 +456,37 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
         helper_bar(); // cold list complete; headers of block b+1 staged
         if (!hdr_warp && !slow) {
             // ---- S3b: hash the cold non-zeros, one per thread and pass
-            const int n_cold = st.n_cold;
+            const int n_cold = lds_s32(a_ncold);
             for (int i0 = 0; i0 < n_cold; i0 += kEntryThreads) {
                 const int i = i0 + et;
                 bool is_new = false;
                 uint32_t p = 0;
                 if (i < n_cold) {
-                    const uint32_t je = st.cold[i];
+                    const uint32_t je = lds_u16(a_cold + 2u * i);
                     const int j = je >> 8, e = je & 255;
-                    const int32_t idx = st.idx[j][st.shift[q][j] + e];
+                    const int32_t idx = lds_s32(a_sidx + kStageRow * j + 4u * (lds_s32(a_shiftq + 4u * j) + e));
                     p = hash_slot<HTC>(idx);
                     bool placed = false;
-                    if (B.n_occ <= kMaxOcc) {
+                    if (lds_s32(a_nocc) <= kMaxOcc) {
                         for (int probe = 0; probe < HTC; ++probe) {
                             // a plain read settles most probes; only an empty slot needs the compare-and-swap
-                            int32_t seen = *reinterpret_cast<volatile int32_t *>(&B.key[p]);
-                            if (seen == -1) seen = atomicCAS(&B.key[p], -1, idx);
+                            int32_t seen = lds_s32(a_key + 4u * p);
+                            if (seen == -1) seen = atoms_cas(a_key + 4u * p, -1, idx);
                             if (seen == -1) { is_new = true; placed = true; break; }
                             if (seen == idx) { placed = true; break; }
                             p = (p + 1) & (HTC - 1);
                         }
                     }
                     if (!placed) { B.slow = 2; p = 0; } // over-full: the block will be walked unstaged
-                    B.pos[j][e] = (uint16_t)(HOT + q * HTC + p);
+                    sts_u16(a_bpos + (uint32_t)(2 * CAP) * j + 2u * e, (uint32_t)(HOT + q * HTC + p));
                 }
                 const uint32_t m = __ballot_sync(0xffffffffu, is_new);
                 if (m) {
                     const int leader = __ffs(m) - 1;
                     int slot = 0;
-                    if (lane == leader) slot = atomicAdd(&B.n_occ, __popc(m));
+                    if (lane == leader) slot = atoms_add(a_nocc, __popc(m));
                     slot = __shfl_sync(0xffffffffu, slot, leader) + __popc(m & lt_mask);
-                    if (is_new) B.occ[slot & (HTC - 1)] = (uint16_t)p;
+                    if (is_new) sts_u16(a_occ + 2u * (slot & (HTC - 1)), p);
                 }
             }
         }
@@ -486,7 +496,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
         if (!slow && (B.slow == 2 || B.n_occ > kMaxOcc)) slow = true;
         if (!slow) {
             // ---- S3c: per distinct cold id: v, a look-up in the previous table, and w_local if U_k is final
-            const int n_occ = B.n_occ;
+            const int n_occ = lds_s32(a_nocc);
             for (int base = 0; base < n_occ; base += 2 * kHelperThreads) {
                 uint32_t pp[2];
                 float vv[2], uu[2];
@@ -498,19 +508,19 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                     fetch[r] = false;
                     vv[r] = uu[r] = 0.0f;
                     if (i >= n_occ) continue;
-                    const uint32_t p = B.occ[i];
-                    const int32_t idx = B.key[p];
-                    uint16_t cp = kNoCarry;
+                    const uint32_t p = lds_u16(a_occ + 2u * i);
+                    const int32_t idx = lds_s32(a_key + 4u * p);
+                    uint32_t cp = kNoCarry;
                     if (have_prev && !prev_slow) {
                         uint32_t r2 = hash_slot<HTC>(idx);
                         for (int probe = 0; probe < HTC; ++probe) {
-                            const int32_t kr = Prev.key[r2];
-                            if (kr == idx) { cp = (uint16_t)r2; break; }
+                            const int32_t kr = lds_s32(a_keyp + 4u * r2);
+                            if (kr == idx) { cp = r2; break; }
                             if (kr == -1) break;
                             r2 = (r2 + 1) & (HTC - 1);
                         }
                     }
-                    B.carry[p] = cp;
+                    sts_u16(a_carry + 2u * p, cp);
                     pp[r] = p;
                     vv[r] = P.vbase[idx];
                     fetch[r] = cp == kNoCarry && early_ok;
@@ -519,8 +529,8 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
 #pragma unroll
                 for (int r = 0; r < 2; ++r)
                     if (pp[r] < HTC) {
-                        B.Tv[pp[r]] = vv[r];
-                        if (fetch[r]) Tw[pp[r]] = fmaf(P.sigma, uu[r], vv[r]);
+                        sts_f32(a_tv + 4u * pp[r], vv[r]);
+                        if (fetch[r]) sts_f32(a_tw + 4u * pp[r], fmaf(P.sigma, uu[r], vv[r]));
                     }
             }
         }
@@ -536,21 +546,21 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
         }
         // ---- S7: complete the table: carried slots from the previous table, late fetches
         if (!slow) {
-            const int n_occ = B.n_occ;
+            const int n_occ = lds_s32(a_nocc);
             for (int base = 0; base < n_occ; base += 4 * kHelperThreads) {
-                uint32_t pp[4];
-                uint16_t cc[4];
+                uint32_t pp[4], cc[4];
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
                     const int i = base + r * kHelperThreads + ht;
-                    pp[r] = i < n_occ ? B.occ[i] : HTC;
+                    pp[r] = i < n_occ ? lds_u16(a_occ + 2u * i) : HTC;
                 }
 #pragma unroll
-                for (int r = 0; r < 4; ++r) cc[r] = pp[r] < HTC ? B.carry[pp[r]] : kNoCarry;
+                for (int r = 0; r < 4; ++r) cc[r] = pp[r] < HTC ? lds_u16(a_carry + 2u * pp[r]) : kNoCarry;
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
-                    if (cc[r] != kNoCarry) Tw[pp[r]] = TwPrev[cc[r]];
-                    else if (!early_ok && pp[r] < HTC) Tw[pp[r]] = fmaf(P.sigma, __ldcg(Uk + B.key[pp[r]]), B.Tv[pp[r]]);
+                    if (cc[r] != kNoCarry) sts_f32(a_tw + 4u * pp[r], lds_f32(a_twp + 4u * cc[r]));
+                    else if (!early_ok && pp[r] < HTC)
+                        sts_f32(a_tw + 4u * pp[r], fmaf(P.sigma, __ldcg(Uk + lds_s32(a_key + 4u * pp[r])), lds_f32(a_tv + 4u * pp[r])));
                 }
             }
         }
@@ -607,6 +617,8 @@ template <int LOSS, bool DENSE, int HOT, int HTC, int CAP> cudaError_t launch_on
 
 // skewed ids (most non-zeros fall on a few thousand ids): a large direct array and a small table
 constexpr int kHotA = 24576, kHtcA = 1024, kCapA = 96;
+// the same for data whose coordinates are often longer than 96 entries: a smaller direct array buys room for them
+constexpr int kHotA2 = 20480, kHtcA2 = 1024, kCapA2 = 128;
 // flat ids: no direct array, everything through the table
 constexpr int kHotB = 0, kHtcB = 4096, kCapB = 128;
 // short dense rows: entry e of every row is id e, all of w_local is "hot", no table
@@ -615,13 +627,15 @@ constexpr int kHotD = 128, kHtcD = 32, kCapD = 128;
 template <int LOSS> cudaError_t launch_loss(Glm &g, const SolverParams &P)
 {
     if (g.fmt == CHICLE_FMT_DENSE_ROWMAJOR) return launch_one<LOSS, true, kHotD, kHtcD, kCapD>(g, P);
-    if (g.hot_variant) return launch_one<LOSS, false, kHotA, kHtcA, kCapA>(g, P);
+    if (g.hot_variant == 1) return launch_one<LOSS, false, kHotA, kHtcA, kCapA>(g, P);
+    if (g.hot_variant == 2) return launch_one<LOSS, false, kHotA2, kHtcA2, kCapA2>(g, P);
     return launch_one<LOSS, false, kHotB, kHtcB, kCapB>(g, P);
 }
 
 } // namespace
 
 int blocked_solver_hot_ids() { return kHotA; }
+int blocked_solver_short_cap() { return kCapA; }
 int blocked_solver_max_dense_dim() { return kCapD; }
 
 cudaError_t launch_blocked_solver(Glm &g, const SolverParams &P)

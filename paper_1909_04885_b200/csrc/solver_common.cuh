@@ -53,6 +53,33 @@ __device__ __forceinline__ void sts_f32(uint32_t a, float v)
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
 }
 
+__device__ __forceinline__ int32_t lds_s32(uint32_t a)
+{
+    int32_t v;
+    asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_s32(uint32_t a, int32_t v)
+{
+    asm volatile("st.shared.s32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts_u16(uint32_t a, uint32_t v)
+{
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"((uint16_t)v) : "memory");
+}
+__device__ __forceinline__ int32_t atoms_cas(uint32_t a, int32_t expect, int32_t v)
+{
+    int32_t old;
+    asm volatile("atom.shared.cas.b32 %0, [%1], %2, %3;" : "=r"(old) : "r"(a), "r"(expect), "r"(v) : "memory");
+    return old;
+}
+__device__ __forceinline__ int32_t atoms_add(uint32_t a, int32_t v)
+{
+    int32_t old;
+    asm volatile("atom.shared.add.s32 %0, [%1], %2;" : "=r"(old) : "r"(a), "r"(v) : "memory");
+    return old;
+}
+
 // Sum over the warp through a 32-float shared-memory buffer: every lane stores its partial, then reads all 32 with
 // eight 128-bit loads and adds them in a fixed tree. About 100 cycles against about 150 for five shuffle rounds.
 // `buf` must be 16-byte aligned; the caller separates successive uses with __syncwarp().
