@@ -85,7 +85,8 @@ typedef struct {
     float ms_reduce;      /* a5: v += sum_k dv_k                                                */
     float ms_total;       /* whole round                                                        */
     int64_t steps;        /* coordinate steps taken in this round, all partitions               */
-    int32_t solver_variant; /* 0 dense ring, 1 sparse blocked, 2 sparse ring, 3 dense blocked (rows <= 128) */
+    int32_t solver_variant; /* 0 dense ring, 1 sparse blocked, 2 sparse ring, 3 dense blocked (rows <= 128),
+                               4 sparse look-ahead, 5 dense look-ahead (rows <= 128) */
     int32_t reserved;
 } chicle_round_stats_t;
 

@@ -323,6 +323,24 @@ chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed)
         dev_free(h, h->part_off);
         delete[] h->h_part_off;
         U = newU; part_off = new_off; h_off = new_hoff;
+        // the look-ahead solver's per-round records (their number depends on K); without them the blocked solver runs
+        dev_free(h, h->la_rec); dev_free(h, h->la_dir); dev_free(h, h->la_cursor);
+        h->la_rec = nullptr; h->la_dir = nullptr; h->la_cursor = nullptr; h->la_rec_bytes = 0;
+        const bool dense_fmt = h->fmt == CHICLE_FMT_DENSE_ROWMAJOR;
+        if (!dense_fmt || h->dim <= lookahead_max_dense_dim()) {
+            size_t rec_bytes = 0, dir_bytes = 0;
+            lookahead_workspace(n, h->nnz, K, dense_fmt, h->dim, &rec_bytes, &dir_bytes);
+            unsigned char *rec = nullptr, *dir = nullptr;
+            if (alloc_into(h, rec, rec_bytes) && alloc_into(h, dir, dir_bytes) && alloc_into(h, h->la_cursor, 16)) {
+                h->la_rec = rec;
+                h->la_dir = dir;
+                h->la_rec_bytes = rec_bytes;
+                (void)cudaMemsetAsync(h->la_cursor, 0, 16 * sizeof(unsigned long long), h->stream);
+            } else {
+                dev_free(h, rec); dev_free(h, dir); dev_free(h, h->la_cursor);
+                h->la_cursor = nullptr;
+            }
+        }
     }
     if (fresh) { h->owner = owner; h->members = members; h->perm = perm; h->perm_epochs = 1; }
     h->U = U; h->part_off = part_off; h->h_part_off = h_off;

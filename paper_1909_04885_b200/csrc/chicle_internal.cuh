@@ -52,6 +52,8 @@ cudaError_t radix_pass(const uint64_t *keys_in, const int32_t *vals_in, uint64_t
                        const int32_t *owner, int64_t n, int shift, uint32_t *hist, uint32_t *scan_sums,
                        cudaStream_t stream);
 
+struct SolverParams;
+
 // ---- handle -------------------------------------------------------------------------------------------------
 struct Glm {
     int device = 0;
@@ -93,6 +95,13 @@ struct Glm {
     float *U = nullptr;         // K * dim: per-partition accumulated update, zero between rounds
     int64_t U_rows = 0;
 
+    // look-ahead solver: the per-block records that its prepare kernel writes every round, and where each one is
+    // (nullptr when they could not be allocated: the blocked solver runs instead)
+    void *la_rec = nullptr;
+    void *la_dir = nullptr;
+    unsigned long long *la_cursor = nullptr;
+    size_t la_rec_bytes = 0;
+
     SortWorkspace sortws;
     double *gap_partials = nullptr; // gap kernel partial sums
     int gap_blocks = 0;
@@ -121,6 +130,9 @@ cudaError_t launch_refresh_resid(Glm &g);                                 // rid
 cudaError_t launch_frequency_remap(Glm &g, uint32_t *counts, uint64_t *keys[2], int32_t *vals[2], uint32_t *hist,
                                    uint32_t *scan_sums, int64_t hot_ids, int32_t long_len, unsigned long long *mass);
 cudaError_t launch_gather_f32(Glm &g, const float *src, const int32_t *map, int64_t n, float *dst); // dst[i] = src[map[i]]
+cudaError_t launch_lookahead_solver(Glm &g, const struct SolverParams &P);
+void lookahead_workspace(int64_t n_coord, int64_t nnz, int32_t K, bool dense, int64_t dim, size_t *rec_bytes, size_t *dir_bytes);
+int lookahead_max_dense_dim();
 int blocked_solver_hot_ids();
 int blocked_solver_short_cap();
 

@@ -394,6 +394,11 @@ cudaError_t launch_local_solver(Glm &g, int64_t H, float sigma_prime, int *varia
     int cap, nslot = 64; // a multiple of the producer warp count; each producer owns nslot / P slots
     const char *force = getenv("CHICLE_FORCE_VARIANT"); // debugging aid: "ring" selects the unblocked solver
     const bool ring = force && strcmp(force, "ring") == 0;
+    const bool blocked = force && strcmp(force, "blocked") == 0;
+    if (g.la_rec && !P.multi_epoch && !ring && !blocked && (!dense || g.dim <= lookahead_max_dense_dim())) {
+        *variant = dense ? 5 : 4;
+        return launch_lookahead_solver(g, P);
+    }
     if (dense && g.dim <= blocked_solver_max_dense_dim() && !ring) {
         *variant = 3;
         return launch_blocked_solver(g, P);

@@ -188,9 +188,31 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
+// a' = sigmoid(z) at the root of z + q sigmoid(z) = c: the root is taken on the convex branch z <= 0 (a positive root
+// is reflected first), Newton from a Lambert-W-like start, fixed iteration count.
+__device__ __forceinline__ float logistic_root(float c, float q)
+{
+    const bool flip = c > 0.5f * q;
+    if (flip) c = q - c;
+    const float kappa = q > 0.0f ? __logf(q) + c : -CUDART_INF_F;
+    float z = kappa <= 0.0f ? fminf(c, 0.0f) : fminf(c - (kappa - __logf(1.0f + kappa)), 0.0f);
+#pragma unroll
+    for (int it = 0; it < kNewtonIters; ++it) {
+        const float e = __expf(z);
+        const float r = __frcp_rn(1.0f + e);
+        const float p = e * r;
+        const float F = fmaf(q, p, z) - c;
+        const float Fp = fmaf(q * p, r, 1.0f); // 1 + q p (1 - p), 1 - p = 1 / (1 + e)
+        z = fminf(z - __fdividef(F, Fp), 0.0f);
+    }
+    const float e = __expf(z);
+    const float r = __frcp_rn(1.0f + e);
+    return flip ? r : e * r;
+}
+
 // Scalar steps. `dot` is x_c . v_local (dual) or c_j . (v_local - y) (ridge). Returns delta and the new state.
-template <int LOSS>
-__device__ __forceinline__ void coordinate_step(float dot, const SlotHdr &h, float &delta, float &new_state)
+template <int LOSS, class Hdr>
+__device__ __forceinline__ void coordinate_step(float dot, const Hdr &h, float &delta, float &new_state)
 {
     if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
         // p0 = 1/n, p1 = w_j, p2 = 1 / (sigma' |c_j|^2 / n + lambda), p3 = lambda
@@ -206,27 +228,8 @@ __device__ __forceinline__ void coordinate_step(float dot, const SlotHdr &h, flo
         new_state = h.p3 * a_new;
     } else {
         // logistic: p0 = y / (lambda n), p1 = a, p2 = q = sigma' |x|^2 / (lambda n), p3 = y.
-        // Root of z + q sigmoid(z) = c on its convex branch (after reflecting a positive root), Newton from a
-        // Lambert-W-like start, fixed iteration count.
         const float q = h.p2, a = h.p1;
-        const float m = dot * h.p0;
-        float c = fmaf(q, a, -m);
-        const bool flip = c > 0.5f * q;
-        if (flip) c = q - c;
-        const float kappa = q > 0.0f ? __logf(q) + c : -CUDART_INF_F;
-        float z = kappa <= 0.0f ? fminf(c, 0.0f) : fminf(c - (kappa - __logf(1.0f + kappa)), 0.0f);
-#pragma unroll
-        for (int it = 0; it < kNewtonIters; ++it) {
-            const float e = __expf(z);
-            const float r = __frcp_rn(1.0f + e);
-            const float p = e * r;
-            const float F = fmaf(q, p, z) - c;
-            const float Fp = fmaf(q * p, r, 1.0f); // 1 + q p (1 - p), 1 - p = 1 / (1 + e)
-            z = fminf(z - __fdividef(F, Fp), 0.0f);
-        }
-        const float e = __expf(z);
-        const float r = __frcp_rn(1.0f + e);
-        const float a_new = flip ? r : e * r;
+        const float a_new = logistic_root(fmaf(q, a, -(dot * h.p0)), q);
         delta = h.p3 * (a_new - a);
         new_state = h.p3 * a_new;
     }

@@ -191,6 +191,56 @@ def test_device_resident_inputs_and_plain_cuda_allocator_give_the_same_bits():
         assert np.array_equal(r[0], res[0][0]) and np.array_equal(r[1], res[0][1]) and r[2] == res[0][2]
 
 
+# ------------------------------------------------------------------ solver families
+@pytest.mark.parametrize("variant", ["blocked"])
+def test_older_solvers_still_match(variant, monkeypatch):
+    # single-epoch rounds take the look-ahead solver by default; the blocked solver stays selectable
+    monkeypatch.setenv("CHICLE_FORCE_VARIANT", variant)
+    run_parity(datagen.make("hinge_csr", 100), rounds=4)
+    run_parity(datagen.make("ridge_csc", 100), rounds=3)
+    run_parity(tiny_dense(500, 28, seed=2, loss="logistic", K=4))
+
+
+def test_lookahead_solver_is_the_default_for_single_epoch_rounds():
+    for w, want in ((datagen.make("hinge_csr", 100), 4), (datagen.make("hinge_dense", 4), 5)):
+        glm = binding.from_workload(w)
+        try:
+            glm.partition(w.phases[0].K, 0)
+            assert glm.cocoa_round(0, float(w.phases[0].K), stats=True)["solver_variant"] == want
+            assert glm.cocoa_round(5, float(w.phases[0].K), stats=True)["solver_variant"] == want
+            n_k = w.n_coord // w.phases[0].K
+            assert glm.cocoa_round(2 * n_k, float(w.phases[0].K), stats=True)["solver_variant"] in (1, 3)
+        finally:
+            glm.close()
+
+
+def test_lookahead_blocks_that_do_not_fit_are_walked_in_place():
+    # rows longer than a staged row (128 entries) and a block with more distinct ids than the buffers hold
+    run_parity(tiny_csr(200, 3000, seed=9, K=2, density=0.03, long_row=500))
+    rng = np.random.default_rng(4)
+    n, d = 256, 40000
+    indptr = np.arange(n + 1, dtype=np.int64) * 120
+    idx = np.concatenate([np.sort(rng.choice(d, 120, replace=False)) for _ in range(n)]).astype(np.int32)
+    vals = rng.standard_normal(n * 120).astype(np.float32) * 0.1
+    y = np.where(rng.random(n) < 0.5, 1.0, -1.0).astype(np.float32)
+    run_parity(Workload("wide_blocks", "hinge", "csr", n, d, vals, y, 1.0 / n, 3, [Phase(0, 2, 0, 2.0)], indptr, idx))
+
+
+def test_lookahead_runs_are_bit_reproducible():
+    w = datagen.make("hinge_csr", 100)
+    res = []
+    for _ in range(2):
+        glm = binding.from_workload(w)
+        try:
+            glm.partition(16, 0)
+            for _ in range(3):
+                glm.cocoa_round(0, 16.0)
+            res.append((glm.get_alpha().copy(), glm.get_v().copy()))
+        finally:
+            glm.close()
+    assert np.array_equal(res[0][0], res[1][0]) and np.array_equal(res[0][1], res[1][1])
+
+
 def test_round_stats():
     w = datagen.make("hinge_csr", 100)
     glm = binding.from_workload(w)
