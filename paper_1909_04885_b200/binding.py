@@ -47,7 +47,7 @@ class Allocator(C.Structure):
 
 class RoundStats(C.Structure):
     _fields_ = [("ms_permutation", C.c_float), ("ms_local", C.c_float), ("ms_reduce", C.c_float), ("ms_total", C.c_float),
-                ("steps", C.c_int64), ("solver_variant", C.c_int32), ("reserved", C.c_int32)]
+                ("steps", C.c_int64), ("solver_variant", C.c_int32), ("ms_prepare", C.c_float)]
 
 
 _lib = None
@@ -213,7 +213,8 @@ class Glm:
             rs = RoundStats()
             self._check(self._lib.chicle_cocoa_round(self._h, H, C.c_float(sp), C.byref(rs)))
             return {"ms_permutation": rs.ms_permutation, "ms_local": rs.ms_local, "ms_reduce": rs.ms_reduce,
-                    "ms_total": rs.ms_total, "steps": rs.steps, "solver_variant": rs.solver_variant}
+                    "ms_total": rs.ms_total, "steps": rs.steps, "solver_variant": rs.solver_variant,
+                    "ms_prepare": rs.ms_prepare}
         self._check(self._lib.chicle_cocoa_round(self._h, H, C.c_float(sp), None))
         return None
 

@@ -385,6 +385,7 @@ chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime
     if (e != cudaSuccess) return fail_cuda(h, e, "visiting-order kernels");
     if (stats) (void)cudaEventRecord(h->ev[1], s);
     int variant = 0;
+    h->time_prepare = stats != nullptr;
     e = launch_local_solver(*h, H, sigma_prime, &variant);
     if (e != cudaSuccess) return fail_cuda(h, e, "local solver launch");
     if (stats) (void)cudaEventRecord(h->ev[2], s);
@@ -408,6 +409,7 @@ chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime
         }
         r.steps = steps;
         r.solver_variant = variant;
+        if (variant >= 4) (void)cudaEventElapsedTime(&r.ms_prepare, h->ev[1], h->ev[4]);
         *stats = r;
     }
     return CHICLE_OK;

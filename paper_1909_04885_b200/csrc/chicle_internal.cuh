@@ -101,6 +101,7 @@ struct Glm {
     void *la_dir = nullptr;
     unsigned long long *la_cursor = nullptr;
     size_t la_rec_bytes = 0;
+    bool time_prepare = false; // record ev[4] between the prepare and the chain kernel (round statistics asked for)
 
     SortWorkspace sortws;
     double *gap_partials = nullptr; // gap kernel partial sums

@@ -48,7 +48,8 @@ constexpr int kLB = 32;          // steps per block
 constexpr int kCapL = 128;       // longest coordinate a staged block can hold
 constexpr int kMaxNz = kLB * kCapL;
 constexpr int kHT = 4096;        // slots of the prepare kernel's hash table (>= kMaxNz)
-constexpr int kPreThreads = 256;
+constexpr int kPreThreads = 256;  // dense prepare kernel
+constexpr int kPreThreadsS = 512; // sparse prepare kernel
 constexpr int kChainThreads = 512;
 constexpr int kChainWarps = kChainThreads / 32;
 constexpr int kRowsPerWarp = kLB / kChainWarps;
@@ -224,14 +225,14 @@ struct PreShared {
     int64_t rs[kLB];
     int32_t nnz[kLB];
     int32_t roff[kLB + 1];
-    uint32_t warp_tot[kPreThreads / 32];
+    uint32_t warp_tot[kPreThreadsS / 32];
     float gsc[kLB], ys[kLB], as[kLB]; // per coordinate: its Gram scale, and what multiplies / enters from the earlier ones
     int32_t n_distinct, total, too_long;
     uint32_t bytes;
     unsigned long long offset;
 };
 
-template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_prepare(const LookParams P)
+template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahead_prepare(const LookParams P)
 {
     extern __shared__ __align__(16) unsigned char smem_pre[];
     PreShared &sh = *reinterpret_cast<PreShared *>(smem_pre);
@@ -273,7 +274,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
             sh.n_distinct = 0;
         }
     }
-    for (int p = tid; p < kHT; p += kPreThreads) {
+    for (int p = tid; p < kHT; p += kPreThreadsS) {
         sh.key[p] = -1;
         sh.mask[p] = 0u;
     }
@@ -282,7 +283,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
     bool slow = sh.too_long != 0;
     if (!slow) {
         // ---- the block's non-zeros into shared memory, every id into the table
-        for (int j = warp; j < cnt; j += kPreThreads / 32) {
+        for (int j = warp; j < cnt; j += kPreThreadsS / 32) {
             const int n = sh.nnz[j], r0 = sh.roff[j];
             const int64_t rs = sh.rs[j];
             for (int e = lane; e < n; e += 32) {
@@ -310,7 +311,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
     //      of the threads before it
     uint32_t mine = 0;
     if (!slow)
-        for (int p = tid; p < kHT; p += kPreThreads) {
+        for (int p = tid; p < kHT; p += kPreThreadsS) {
             const uint32_t m = sh.mask[p];
             if (m & (m - 1u)) mine += (1u << 16) + (uint32_t)__popc(m);
         }
@@ -323,7 +324,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
     if (lane == 31) sh.warp_tot[warp] = incl;
     __syncthreads();
     uint32_t run = incl - mine, all = 0;
-    for (int w2 = 0; w2 < kPreThreads / 32; ++w2) {
+    for (int w2 = 0; w2 < kPreThreadsS / 32; ++w2) {
         if (w2 < warp) run += sh.warp_tot[w2];
         all += sh.warp_tot[w2];
     }
@@ -359,7 +360,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
     int32_t *ids_g = idx_g + total;
     uint16_t *cpos_g = reinterpret_cast<uint16_t *>(ids_g + T);
     uint16_t *off_g = cpos_g + total;
-    for (int p = tid; p < kHT; p += kPreThreads) {
+    for (int p = tid; p < kHT; p += kPreThreadsS) {
         const uint32_t m = sh.mask[p];
         if (m & (m - 1u)) {
             const uint32_t t = run >> 16, o = run & 0xffffu;
@@ -372,7 +373,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
     if (tid == 0) off_g[T] = (uint16_t)total_m;
     __syncthreads();
     // ---- list entries: a non-zero's place in its id's list is the number of lower coordinates that have the id
-    for (int j = warp; j < cnt; j += kPreThreads / 32) {
+    for (int j = warp; j < cnt; j += kPreThreadsS / 32) {
         const int n = sh.nnz[j], r0 = sh.roff[j];
         for (int e = lane; e < n; e += 32) {
             const int p = sh.slot[r0 + e];
@@ -386,21 +387,40 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
             val_g[r0 + e] = sh.val[r0 + e];
             idx_g[r0 + e] = sh.idx[r0 + e] | (shared_id ? (int32_t)0x80000000 : 0);
             cpos_g[r0 + e] = (uint16_t)pos;
+            // for the Gram pass: the id itself is no longer needed, its mask and its list's start are
+            sh.idx[r0 + e] = (int32_t)m;
+            sh.slot[r0 + e] = sh.soff[p];
         }
     }
     __syncthreads();
-    // ---- Gram triangle: a warp per coordinate j, lane l collects x_j . x_l over j's entries in ascending order
-    for (int j = warp; j < kLB; j += kPreThreads / 32) {
+    // ---- Gram triangle: a warp per coordinate j, lane l collects x_j . x_l over j's entries in ascending order. The
+    //      lanes first look at 32 entries at once and keep those whose id an earlier coordinate has too; only these
+    //      are then walked, their mask, list start and value handed round by shuffles.
+    for (int j = warp; j < kLB; j += kPreThreadsS / 32) {
         float acc = 0.0f;
         if (j < cnt) {
             const int n = sh.nnz[j], r0 = sh.roff[j];
-            const uint32_t below = (1u << j) - 1u;
-            for (int e = 0; e < n; ++e) {
-                const int p = sh.slot[r0 + e];
-                const uint32_t m = sh.mask[p];
-                if ((m & below) == 0u) continue; // no earlier coordinate has this id (same for the whole warp)
-                if ((m >> lane) & 1u & (lane < j ? 1u : 0u))
-                    acc = fmaf(sh.val[r0 + e], sh.val[sh.ent[sh.soff[p] + __popc(m & ((1u << lane) - 1u))]], acc);
+            const uint32_t below = (1u << j) - 1u, lt = (1u << lane) - 1u;
+            const bool mine = lane < j;
+            for (int e0 = 0; e0 < n; e0 += 32) {
+                const int e = e0 + lane;
+                uint32_t m_l = 0u;
+                int so_l = 0;
+                float x_l = 0.0f;
+                if (e < n) {
+                    m_l = (uint32_t)sh.idx[r0 + e];
+                    so_l = sh.slot[r0 + e];
+                    x_l = sh.val[r0 + e];
+                }
+                uint32_t todo = __ballot_sync(0xffffffffu, (m_l & below) != 0u);
+                while (todo) {
+                    const int src = __ffs(todo) - 1;
+                    todo &= todo - 1u;
+                    const uint32_t m = __shfl_sync(0xffffffffu, m_l, src);
+                    const int so = __shfl_sync(0xffffffffu, so_l, src);
+                    const float x = __shfl_sync(0xffffffffu, x_l, src);
+                    if (((m >> lane) & 1u) && mine) acc = fmaf(x, sh.val[sh.ent[so + __popc(m & lt)]], acc);
+                }
             }
         }
         acc *= sh.gsc[j] * sh.ys[lane];
@@ -411,7 +431,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
         if (lane == 0 && j < cnt) out.hdr[j].q0 = q0;
     }
     __syncthreads();
-    for (int i = tid; i < kLB * kLB; i += kPreThreads) out.G[i] = sh.G[i >> 5][i & 31];
+    for (int i = tid; i < kLB * kLB; i += kPreThreadsS) out.G[i] = sh.G[i >> 5][i & 31];
 }
 
 // Short dense rows: every row has every id, so the lists are implicit: headers, Gram triangle and the rows.
@@ -887,14 +907,16 @@ template <int LOSS> cudaError_t launch_loss(Glm &g, LookParams &P)
         k_lookahead_prepare_dense<LOSS><<<nb, kPreThreads, 0, g.stream>>>(P);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
+        if (g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
         return launch_chain<LOSS, true, kCapL, 4, 4>(g, P);
     }
     auto pre = k_lookahead_prepare<LOSS>;
     e = cudaFuncSetAttribute(pre, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PreShared));
     if (e != cudaSuccess) return e;
-    pre<<<nb, kPreThreads, sizeof(PreShared), g.stream>>>(P);
+    pre<<<nb, kPreThreadsS, sizeof(PreShared), g.stream>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
     if (g.hot_variant) return launch_chain<LOSS, false, kHotSkew, kTmax, 2>(g, P);
     return launch_chain<LOSS, false, 4, kTmax, 4>(g, P);
 }
