@@ -5,8 +5,8 @@
 // The walk is cut into blocks of 32 consecutive steps. Inside a block, with w the local model at the block's start,
 //     dot_j = x_j . w + sigma' * sum_{l < j} delta_l * (x_j . x_l),
 // so once the 32 dot products against w and the strictly lower triangle of the block's Gram matrix G_jl = x_j . x_l
-// are known, the 32 steps are a scalar recurrence: one warp, lane j owns coordinate j, and a step costs the scalar
-// map, one shuffle that broadcasts its result, and one fused multiply-add per lane. The block then applies
+// are known, the 32 steps are a scalar recurrence run by one warp: a step costs the scalar map and a few fused
+// multiply-adds, plus one shuffle per coordinate to hand the results round. The block then applies
 // w += sigma' * sum_j delta_j x_j in parallel. Which coordinates meet in a block is fixed by the visiting order
 // alone, not by the model, so everything structural is prepared for all blocks of all partitions at once by a
 // throughput kernel that uses the whole GPU, and the latency-bound kernel (one CTA per partition) only consumes it.
@@ -227,7 +227,7 @@ struct PreShared {
     int32_t roff[kLB + 1];
     uint32_t warp_tot[kPreThreadsS / 32];
     float gsc[kLB], ys[kLB], as[kLB]; // per coordinate: its Gram scale, and what multiplies / enters from the earlier ones
-    int32_t n_distinct, total, too_long;
+    int32_t total, too_long;
     uint32_t bytes;
     unsigned long long offset;
 };
@@ -271,7 +271,6 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
             sh.roff[kLB] = incl;
             sh.total = incl;
             sh.too_long = too_long ? 1 : 0;
-            sh.n_distinct = 0;
         }
     }
     for (int p = tid; p < kHT; p += kPreThreadsS) {
@@ -295,7 +294,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
                     int32_t seen = sh.key[p];
                     if (seen == -1) {
                         seen = atomicCAS(&sh.key[p], -1, id);
-                        if (seen == -1) { atomicAdd(&sh.n_distinct, 1); break; }
+                        if (seen == -1) break;
                     }
                     if (seen == id) break;
                     p = (p + 1) & (kHT - 1);
@@ -553,19 +552,23 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
     __syncthreads();
     if (nblocks == 0) return;
 
-    // ---- warp 1, lane 0: where a block's record is, and the copy itself
-    auto load_dir = [&](int64_t blk) -> BlkDir {
-        BlkDir d{0ull, 0u, 0u};
-        if (blk < nblocks && lane == 0) d = P.dir[bid0 + blk];
-        return d;
+    // ---- warp 1: where a block's record is, and the copy itself. The directory entry of block b + 2 is loaded while
+    //      block b runs and first looked at a block later (an unconditional load from a clamped address, so that
+    //      nothing has to wait for it at the point of issue).
+    auto load_dir = [&](int64_t blk, uint32_t (&d)[4]) {
+        const int64_t at = blk < nblocks ? blk : nblocks - 1;
+        asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+                     : "l"(P.dir + (bid0 + at))
+                     : "memory");
     };
-    auto issue = [&](int64_t blk, const BlkDir &d) {
+    auto issue = [&](int64_t blk, const uint32_t (&d)[4]) {
         if (blk >= nblocks || lane != 0) return;
         const uint32_t bar = smem_u32(&sh.full[blk & 1]);
-        // the buffer was last written by ordinary stores (the products of the update phase): order them before the
-        // copy engine's writes
+        // the buffer was last written by ordinary stores: order them before the copy engine's writes
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        const uint32_t bytes = d.bytes <= Shared::kRecMax ? d.bytes : 0u;
+        const unsigned long long offset = ((unsigned long long)d[1] << 32) | d[0];
+        const uint32_t bytes = d[2] <= Shared::kRecMax ? d[2] : 0u;
         if (bytes == 0) {
             // no record (the prepare kernel ran out of room): nothing will arrive, say so now
             atomicOr(S.status, ST_WAIT_TIMEOUT);
@@ -573,17 +576,18 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
             return;
         }
         mbar_arrive_expect_tx(bar, bytes);
-        bulk_g2s(smem_u32(&sh.rec[blk & 1][0]), P.rec + d.offset, bytes, bar);
+        bulk_g2s(smem_u32(&sh.rec[blk & 1][0]), P.rec + offset, bytes, bar);
     };
-    BlkDir next_dir{0ull, 0u, 0u};
+    uint32_t next_dir[4] = {0u, 0u, 0u, 0u};
     if (warp == 1) {
-        issue(0, load_dir(0));
-        next_dir = load_dir(1);
+        load_dir(0, next_dir);
+        issue(0, next_dir);
+        load_dir(1, next_dir);
     }
 
     bool aborted = false;
 #ifdef CHICLE_LA_TIMING
-    long long tw = 0, tg1 = 0, tg = 0, tr = 0, tp1 = 0, ts = 0, t0 = clock64(), t1 = 0;
+    long long tw = 0, tg1 = 0, tg = 0, tr = 0, tp1 = 0, ts = 0, trw = 0, t0 = clock64(), t1 = 0;
 #endif
     for (int64_t b = 0; b < nblocks; ++b) {
         unsigned char *rec = &sh.rec[b & 1][0];
@@ -599,7 +603,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
         if (slow) {
             if (warp == 1) {
                 issue(b + 1, next_dir);
-                next_dir = load_dir(b + 2);
+                load_dir(b + 2, next_dir);
             }
             if (warp == 0) {
                 // coordinate by coordinate against the model: ids below HOT in shared memory, the rest in row k of
@@ -709,39 +713,78 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
         LA_T(tg);
         // ---------------- (R) the recurrence on warp 0; warp 1 starts the next block's copy meanwhile
         if (warp == 0) {
-            const LookHdr h = H.hdr[lane];
-            float g[kLB];
+            // Four coordinates at a time. Lane q (and its copies q + 8, q + 16, q + 24, which compute the same) keeps
+            // the states of coordinates 4q .. 4q + 3. Group g: its lane walks its four coordinates by itself (no
+            // shuffle inside a group), the four results are handed round, and every lane adds what they mean for
+            // its own four: the step per coordinate costs about half of one shuffle per coordinate.
+            const int q = lane & 7;
+            const float4 *G4 = reinterpret_cast<const float4 *>(H.G); // G4[l * 8 + q]: row l, columns 4q .. 4q + 3
+            LookHdr hh[4];
+            float s[4], mine[4];
 #pragma unroll
-            for (int l = 0; l < kLB; ++l) g[l] = H.G[l * kLB + lane];
-            float s = recurrence_start<LOSS>(sh.m0[lane], h);
-            float mine = 0.0f;
+            for (int i = 0; i < 4; ++i) {
+                hh[i] = H.hdr[4 * q + i];
+                s[i] = recurrence_start<LOSS>(sh.m0[4 * q + i], hh[i]);
+                mine[i] = 0.0f;
+            }
 #pragma unroll
-            for (int l = 0; l < kLB; ++l) {
-                const float out = recurrence_map<LOSS>(s, h); // every lane for its own coordinate; lane l's is final now
-                if (lane == l) mine = out;
-                s = fmaf(__shfl_sync(0xffffffffu, out, l), g[l], s); // g[l] is 0 for l >= lane
-            }
-            float my_delta = 0.0f;
-            if (lane < cnt) {
-                float my_state;
-                if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
-                    my_delta = mine;
-                    my_state = h.p1 + mine;
-                } else {
-                    my_delta = h.p3 * (mine - h.p1);
-                    my_state = h.p3 * mine;
+            for (int g = 0; g < kLB / 4; ++g) {
+                float4 blk[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) blk[k] = G4[(4 * g + k) * 8 + q];
+                // inside the group (the numbers matter on the lanes with q == g, where blk holds the group's own
+                // triangle; the others run the same instructions on copies)
+                float o[4];
+                o[0] = recurrence_map<LOSS>(s[0], hh[0]);
+                const float t1 = fmaf(o[0], blk[0].y, s[1]);
+                o[1] = recurrence_map<LOSS>(t1, hh[1]);
+                const float t2 = fmaf(o[1], blk[1].z, fmaf(o[0], blk[0].z, s[2]));
+                o[2] = recurrence_map<LOSS>(t2, hh[2]);
+                const float t3 = fmaf(o[2], blk[2].w, fmaf(o[1], blk[1].w, fmaf(o[0], blk[0].w, s[3])));
+                o[3] = recurrence_map<LOSS>(t3, hh[3]);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) mine[i] = q == g ? o[i] : mine[i];
+                float og[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) og[k] = __shfl_sync(0xffffffffu, o[k], g);
+                // (zero entries of the triangle make this a no-op for the groups at or before g, whose states are final)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    s[0] = fmaf(og[k], blk[k].x, s[0]);
+                    s[1] = fmaf(og[k], blk[k].y, s[1]);
+                    s[2] = fmaf(og[k], blk[k].z, s[2]);
+                    s[3] = fmaf(og[k], blk[k].w, s[3]);
                 }
-                if (!(fabsf(my_delta) <= CUDART_MAX_NORMAL_F)) {
-                    atomicOr(S.status, ST_NONFINITE_STEP);
-                    my_delta = 0.0f;
-                    my_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? h.p1 : h.p3 * h.p1;
-                }
-                S.alpha[h.coord] = my_state;
             }
-            sh.dj[lane] = my_delta;
+            if (lane < 8) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int j = 4 * q + i;
+                    const LookHdr &h = hh[i];
+                    float my_delta = 0.0f;
+                    if (j < cnt) {
+                        float my_state;
+                        if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+                            my_delta = mine[i];
+                            my_state = h.p1 + mine[i];
+                        } else {
+                            my_delta = h.p3 * (mine[i] - h.p1);
+                            my_state = h.p3 * mine[i];
+                        }
+                        if (!(fabsf(my_delta) <= CUDART_MAX_NORMAL_F)) {
+                            atomicOr(S.status, ST_NONFINITE_STEP);
+                            my_delta = 0.0f;
+                            my_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? h.p1 : h.p3 * h.p1;
+                        }
+                        S.alpha[h.coord] = my_state;
+                    }
+                    sh.dj[j] = my_delta;
+                }
+            }
+            LA_T(trw);
         } else if (warp == 1) {
             issue(b + 1, next_dir);
-            next_dir = load_dir(b + 2);
+            load_dir(b + 2, next_dir);
         }
         __syncthreads();
         LA_T(tr);
@@ -863,7 +906,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
 #endif
     if (blockIdx.x == 0 && tid == LA_TIMING_TID) {
         unsigned long long *d = P.cursor + 2;
-        d[0] = tw; d[1] = tg1; d[2] = tg; d[3] = tr; d[4] = tp1; d[5] = ts; d[6] = nblocks;
+        d[0] = tw; d[1] = tg1; d[2] = tg; d[3] = tr; d[4] = tp1; d[5] = ts; d[6] = nblocks; d[7] = trw;
     }
 #endif
     if (aborted) {
@@ -893,7 +936,8 @@ template <int LOSS, bool DENSE, int HOT, int TMAX, int NCH> cudaError_t launch_c
     (void)cudaMemcpy(t, P.cursor + 2, sizeof(t), cudaMemcpyDeviceToHost);
     const double nb = t[6] ? (double)t[6] : 1.0;
     fprintf(stderr, "lookahead chain, cycles per block (CTA 0): wait %.0f gather %.0f reduce+bar %.0f recurrence %.0f products %.0f "
-            "lists %.0f (%llu blocks)\n", t[0] / nb, t[1] / nb, t[2] / nb, t[3] / nb, t[4] / nb, t[5] / nb, t[6]);
+            "lists %.0f (%llu blocks); warp 0's recurrence alone %.0f, then waiting for warp 1 %.0f\n", t[0] / nb, t[1] / nb, t[2] / nb,
+            (t[3] + t[7]) / nb, t[4] / nb, t[5] / nb, t[6], t[7] / nb, t[3] / nb);
 #endif
     return e;
 }
