@@ -331,11 +331,11 @@ chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed)
             size_t rec_bytes = 0, dir_bytes = 0;
             lookahead_workspace(n, h->nnz, K, dense_fmt, h->dim, &rec_bytes, &dir_bytes);
             unsigned char *rec = nullptr, *dir = nullptr;
-            if (alloc_into(h, rec, rec_bytes) && alloc_into(h, dir, dir_bytes) && alloc_into(h, h->la_cursor, 16)) {
+            if (alloc_into(h, rec, rec_bytes) && alloc_into(h, dir, dir_bytes) && alloc_into(h, h->la_cursor, 32)) {
                 h->la_rec = rec;
                 h->la_dir = dir;
                 h->la_rec_bytes = rec_bytes;
-                (void)cudaMemsetAsync(h->la_cursor, 0, 16 * sizeof(unsigned long long), h->stream);
+                (void)cudaMemsetAsync(h->la_cursor, 0, 32 * sizeof(unsigned long long), h->stream);
             } else {
                 dev_free(h, rec); dev_free(h, dir); dev_free(h, h->la_cursor);
                 h->la_cursor = nullptr;

@@ -220,7 +220,7 @@ struct PreShared {
     int32_t key[kHT];        // id in a table slot, -1 = empty
     uint32_t mask[kHT];      // bit j: coordinate j of the block has this id
     uint16_t soff[kHT];      // start of the slot's list
-    uint16_t ent[kMaxNz];    // list entries: positions in val
+    float lval[kMaxNz];      // the values of the non-zeros with shared ids, list after list (for the Gram pass)
     float G[kLB][kLB + 1];
     int64_t rs[kLB];
     int32_t nnz[kLB];
@@ -245,6 +245,12 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     const int64_t nk = P.S.part_off[k + 1] - off;
     const int64_t steps = steps_of(P, nk);
     const int cnt = (int)((steps - b * kLB) < kLB ? (steps - b * kLB) : kLB);
+#ifdef CHICLE_LA_TIMING
+    long long pt0 = clock64(), pt1 = 0;
+#define PRE_T(i) do { asm volatile("" ::: "memory"); pt1 = clock64(); if (tid == 0) atomicAdd(P.cursor + 16 + (i), (unsigned long long)(pt1 - pt0)); pt0 = pt1; asm volatile("" ::: "memory"); } while (0)
+#else
+#define PRE_T(i) do { } while (0)
+#endif
 
     // ---- headers (kept in registers of warp 0 until the record's place is known)
     LookHdr hd{0, 0, 0, 0.f, 0.f, 0.f, 0.f, 0.f, {0.f, 0.f, 0.f}};
@@ -278,6 +284,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
         sh.mask[p] = 0u;
     }
     __syncthreads();
+    PRE_T(0);
     const int total = sh.total;
     bool slow = sh.too_long != 0;
     if (!slow) {
@@ -285,10 +292,21 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
         for (int j = warp; j < cnt; j += kPreThreadsS / 32) {
             const int n = sh.nnz[j], r0 = sh.roff[j];
             const int64_t rs = sh.rs[j];
-            for (int e = lane; e < n; e += 32) {
-                const int32_t id = P.S.indices[rs + e];
+            int32_t ids4[kCapL / 32];
+            float vals4[kCapL / 32];
+#pragma unroll
+            for (int c = 0; c < kCapL / 32; ++c) { // all of the row's loads first
+                const int e = lane + 32 * c;
+                ids4[c] = e < n ? P.S.indices[rs + e] : -1;
+                vals4[c] = e < n ? P.S.values[rs + e] : 0.0f;
+            }
+#pragma unroll
+            for (int c = 0; c < kCapL / 32; ++c) {
+                const int e = lane + 32 * c;
+                if (e >= n) continue;
+                const int32_t id = ids4[c];
                 sh.idx[r0 + e] = id;
-                sh.val[r0 + e] = P.S.values[rs + e];
+                sh.val[r0 + e] = vals4[c];
                 uint32_t p = hash_id(id);
                 for (int probe = 0; probe < kHT; ++probe) {
                     int32_t seen = sh.key[p];
@@ -304,6 +322,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
             }
         }
         __syncthreads();
+    PRE_T(1);
     }
     // ---- number the shared ids (those with more than one bit in their mask) and lay out their lists: thread t owns
     //      slots t, t + 256, ...; its running counts (ids in the high half, list entries in the low half) follow those
@@ -322,6 +341,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     }
     if (lane == 31) sh.warp_tot[warp] = incl;
     __syncthreads();
+    PRE_T(2);
     uint32_t run = incl - mine, all = 0;
     for (int w2 = 0; w2 < kPreThreadsS / 32; ++w2) {
         if (w2 < warp) run += sh.warp_tot[w2];
@@ -342,6 +362,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
         P.dir[bid] = d;
     }
     __syncthreads();
+    PRE_T(3);
     if (sh.bytes == 0) return;
     unsigned char *rec = P.rec + sh.offset;
     BlkHead &out = *reinterpret_cast<BlkHead *>(rec);
@@ -371,6 +392,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     }
     if (tid == 0) off_g[T] = (uint16_t)total_m;
     __syncthreads();
+    PRE_T(4);
     // ---- list entries: a non-zero's place in its id's list is the number of lower coordinates that have the id
     for (int j = warp; j < cnt; j += kPreThreadsS / 32) {
         const int n = sh.nnz[j], r0 = sh.roff[j];
@@ -381,7 +403,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
             int pos = 0;
             if (shared_id) {
                 pos = sh.soff[p] + __popc(m & ((1u << j) - 1u));
-                sh.ent[pos] = (uint16_t)(r0 + e);
+                sh.lval[pos] = sh.val[r0 + e];
             }
             val_g[r0 + e] = sh.val[r0 + e];
             idx_g[r0 + e] = sh.idx[r0 + e] | (shared_id ? (int32_t)0x80000000 : 0);
@@ -392,6 +414,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
         }
     }
     __syncthreads();
+    PRE_T(5);
     // ---- Gram triangle: a warp per coordinate j, lane l collects x_j . x_l over j's entries in ascending order. The
     //      lanes first look at 32 entries at once and keep those whose id an earlier coordinate has too; only these
     //      are then walked, their mask, list start and value handed round by shuffles.
@@ -412,15 +435,23 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
                     x_l = sh.val[r0 + e];
                 }
                 uint32_t todo = __ballot_sync(0xffffffffu, (m_l & below) != 0u);
+                // two entries per turn, so that the second one's loads are under way while the first is added
                 while (todo) {
-                    const int src = __ffs(todo) - 1;
+                    const int src0 = __ffs(todo) - 1;
                     todo &= todo - 1u;
-                    const uint32_t m = __shfl_sync(0xffffffffu, m_l, src);
-                    const int so = __shfl_sync(0xffffffffu, so_l, src);
-                    const float x = __shfl_sync(0xffffffffu, x_l, src);
-                    if (((m >> lane) & 1u) && mine) acc = fmaf(x, sh.val[sh.ent[so + __popc(m & lt)]], acc);
+                    const bool two = todo != 0u;
+                    const int src1 = two ? __ffs(todo) - 1 : src0;
+                    todo &= todo - 1u;
+                    const uint32_t m0 = __shfl_sync(0xffffffffu, m_l, src0), m1 = __shfl_sync(0xffffffffu, m_l, src1);
+                    const int so0 = __shfl_sync(0xffffffffu, so_l, src0), so1 = __shfl_sync(0xffffffffu, so_l, src1);
+                    const float x0 = __shfl_sync(0xffffffffu, x_l, src0), x1 = __shfl_sync(0xffffffffu, x_l, src1);
+                    const bool on0 = (m0 >> lane) & 1u, on1 = two && ((m1 >> lane) & 1u);
+                    const float v0 = sh.lval[on0 ? so0 + __popc(m0 & lt) : 0], v1 = sh.lval[on1 ? so1 + __popc(m1 & lt) : 0];
+                    acc = fmaf(x0, on0 ? v0 : 0.0f, acc);
+                    acc = fmaf(x1, on1 ? v1 : 0.0f, acc);
                 }
             }
+            if (!mine) acc = 0.0f;
         }
         acc *= sh.gsc[j] * sh.ys[lane];
         sh.G[lane][j] = acc; // row l, column j
@@ -430,7 +461,9 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
         if (lane == 0 && j < cnt) out.hdr[j].q0 = q0;
     }
     __syncthreads();
+    PRE_T(6);
     for (int i = tid; i < kLB * kLB; i += kPreThreadsS) out.G[i] = sh.G[i >> 5][i & 31];
+    PRE_T(7);
 }
 
 // Short dense rows: every row has every id, so the lists are implicit: headers, Gram triangle and the rows.
@@ -960,6 +993,17 @@ template <int LOSS> cudaError_t launch_loss(Glm &g, LookParams &P)
     pre<<<nb, kPreThreadsS, sizeof(PreShared), g.stream>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+#ifdef CHICLE_LA_TIMING
+    {
+        unsigned long long t[8] = {0};
+        (void)cudaStreamSynchronize(g.stream);
+        (void)cudaMemcpy(t, P.cursor + 16, sizeof(t), cudaMemcpyDeviceToHost);
+        (void)cudaMemset(P.cursor + 16, 0, sizeof(t));
+        fprintf(stderr, "lookahead prepare, cycles per CTA: headers %.0f insert %.0f count %.0f place %.0f number %.0f entries %.0f gram %.0f write %.0f\n",
+                t[0] / (double)nb, t[1] / (double)nb, t[2] / (double)nb, t[3] / (double)nb, t[4] / (double)nb, t[5] / (double)nb,
+                t[6] / (double)nb, t[7] / (double)nb);
+    }
+#endif
     if (g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
     if (g.hot_variant) return launch_chain<LOSS, false, kHotSkew, kTmax, 2>(g, P);
     return launch_chain<LOSS, false, 4, kTmax, 4>(g, P);
