@@ -3,7 +3,10 @@
 // shared vector used when a state is restored.
 #include <math_constants.h>
 
-#include "chicle_internal.cuh"
+#include <cstdlib>
+#include <cstring>
+
+#include "solver_common.cuh"
 
 namespace chicle {
 
@@ -136,7 +139,7 @@ __device__ __forceinline__ double xlogx(double x) { return x > 0.0 ? x * log(x) 
 
 // adds coordinate c's contribution, given its dot product with the shared vector (with v - y for ridge)
 template <int LOSS>
-__device__ __forceinline__ void gap_term(double dot, float label, float state, double lam_n, double &s0, double &s1)
+__device__ __forceinline__ void gap_term(double dot, float label, float state, double inv_lam_n, double &s0, double &s1)
 {
     if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
         const double w = (double)state;
@@ -144,7 +147,7 @@ __device__ __forceinline__ void gap_term(double dot, float label, float state, d
         s1 += w * w;
     } else {
         const double y = (double)label;
-        const double mu = y * dot / lam_n;
+        const double mu = y * dot * inv_lam_n; // (a multiplication: the fp64 division was a third of the streamed kernel's instructions)
         double a = y * (double)state;
         a = a < 0.0 ? 0.0 : (a > 1.0 ? 1.0 : a);
         double l, conj;
@@ -175,6 +178,7 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
 {
     __shared__ double sh[kThreads][2];
     __shared__ double sh2[kWarpsPerBlock][2];
+    const double inv_lam_n = 1.0 / lam_n;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t nw = (int64_t)gridDim.x * kWarpsPerBlock;
     const int64_t gw = (int64_t)blockIdx.x * kWarpsPerBlock + warp;
@@ -250,7 +254,7 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
                 const double d = warp_sum_d(dot[r]);
                 if (lane == r) mine = d;
             }
-            if (owner) gap_term<LOSS>(mine, my_label, my_state, lam_n, s0, s1);
+            if (owner) gap_term<LOSS>(mine, my_label, my_state, inv_lam_n, s0, s1);
         }
     } else if (dim <= 64 && (dim & 3) == 0) {
         // short dense rows: a thread per row, 128-bit loads; a warp's 32 rows are contiguous in memory
@@ -265,7 +269,7 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
                 dot = fma((double)x.z, (double)vec[4 * j4 + 2], dot);
                 dot = fma((double)x.w, (double)vec[4 * j4 + 3], dot);
             }
-            gap_term<LOSS>(dot, labels[c], state[c], lam_n, s0, s1);
+            gap_term<LOSS>(dot, labels[c], state[c], inv_lam_n, s0, s1);
         }
     } else {
         for (int64_t c = gw; c < n_coord; c += nw) {
@@ -273,7 +277,7 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
             double dot = 0.0;
             for (int64_t j = lane; j < dim; j += 32) dot = fma((double)row[j], (double)vec[j], dot);
             dot = warp_sum_d(dot);
-            if (lane == 0) gap_term<LOSS>(dot, labels[c], state[c], lam_n, s0, s1);
+            if (lane == 0) gap_term<LOSS>(dot, labels[c], state[c], inv_lam_n, s0, s1);
         }
     }
     // slice of the shared vector owned by this block
@@ -319,6 +323,232 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
         double tot = 0.0;
         for (int w = 0; w < kWarpsPerBlock; ++w) tot += sh2[w][threadIdx.x - 2];
         partials[(size_t)blockIdx.x * 4 + threadIdx.x] = tot;
+    }
+}
+
+// Sparse formats, streamed: the coordinates of a block's tile lie one after the other in memory, so their indices and
+// values are two contiguous ranges, which a producer warp brings into a three-stage shared-memory ring with bulk
+// copies (16-byte aligned windows; the bytes in flight no longer depend on registers or on how many warps fit). The
+// sixteen consumer warps take R coordinates per tile, 512 / R threads each (every thread a fixed subset of the
+// coordinate's entries, all gathers from the shared vector issued before the first use), and add the partial dot
+// products in a fixed order. A tile whose non-zeros do not fit a stage is read from global memory by the same threads.
+// Gathers from the shared vector are what the warp-per-coordinate kernel is bound by on skewed data (a 32-byte sector
+// of L2 traffic per 4-byte gather: 7 TB/s at config 2), so each block also keeps the first kGapHot entries of the
+// vector in its shared memory (ids are frequency-ranked: they take most of the gathers); the kernel is used when the
+// ids are skewed, one block per SM. Every wait is bounded; when one runs out the status word says so and all roles
+// leave.
+constexpr int kGapStages = 3;
+constexpr int kGapHot = 32768;             // entries of the shared vector staged per block (128 KB)
+constexpr int kGapCapNz = 3584;            // non-zeros a stage holds
+constexpr int kGapStageElems = kGapCapNz + 8; // + the window's alignment slack
+constexpr int kGapConsumers = 512;
+
+// Bounded wait without back-off (try_wait itself parks the thread for a while): every lane calls it, lane 0 polls.
+__device__ __forceinline__ bool gap_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+        ok = 0;
+        for (uint32_t it = 0; it < kSpinLimit; ++it) {
+            if (mbar_try_wait(bar, parity)) { ok = 1; break; }
+            if ((it & 255u) == 255u && *abort_flag) break;
+        }
+        if (!ok && !*abort_flag) {
+            *abort_flag = 1;
+            atomicOr(status, ST_WAIT_TIMEOUT);
+        }
+    }
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+struct GapShared {
+    alignas(16) float vhot[kGapHot];       // the head of the shared vector (ridge: of v - y)
+    alignas(16) int32_t idx[kGapStages][kGapStageElems];
+    alignas(16) float val[kGapStages][kGapStageElems];
+    alignas(8) uint64_t full[kGapStages];  // the stage's copies have landed (or the tile was marked as not staged)
+    alignas(8) uint64_t empty[kGapStages]; // the consumer warps have finished with the stage
+    long long base[kGapStages];            // first element of the stage's window in the global arrays; -1: not staged
+    double sh[kGapConsumers][2];
+    double sh2[kGapConsumers / 32][2];
+    int abort_flag;
+};
+
+template <int LOSS, int R>
+__global__ void __launch_bounds__(kGapConsumers + 32, 1)
+k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices, const float *__restrict__ values,
+             const float *__restrict__ labels, const float *__restrict__ state, const float *__restrict__ vec,
+             int64_t n_coord, int64_t dim, double lam_n, double *__restrict__ partials, uint32_t *status)
+{
+    constexpr int TPR = kGapConsumers / R; // threads per coordinate
+    constexpr int kMaxPer = 8;             // entries a thread keeps in flight
+    extern __shared__ __align__(128) unsigned char gap_smem[];
+    GapShared &sm = *reinterpret_cast<GapShared *>(gap_smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const double inv_lam_n = 1.0 / lam_n;
+    volatile int *abort_flag = &sm.abort_flag;
+    if (tid == 0) {
+        sm.abort_flag = 0;
+        for (int s2 = 0; s2 < kGapStages; ++s2) {
+            mbar_init(smem_u32(&sm.full[s2]), 1);
+            mbar_init(smem_u32(&sm.empty[s2]), kGapConsumers / 32);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    const int hot_n = (int)(dim < kGapHot ? dim : kGapHot);
+    for (int i = tid; i < hot_n; i += kGapConsumers + 32)
+        sm.vhot[i] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? vec[i] - labels[i] : vec[i];
+    __syncthreads();
+    const int64_t ntiles = (n_coord + R - 1) / R;
+    const int64_t first = blockIdx.x, step = gridDim.x;
+    double s0 = 0.0, s1 = 0.0;
+    if (warp == kGapConsumers / 32) {
+        // ------------------------------------------------ producer (the next tile's extent is fetched a tile ahead)
+        int64_t k = 0;
+        auto bounds = [&](int64_t t, int64_t &rs, int64_t &re) {
+            rs = re = 0;
+            if (t < ntiles && lane == 0) {
+                const int64_t c0 = t * R, c1 = (c0 + R < n_coord) ? c0 + R : n_coord;
+                rs = indptr[c0];
+                re = indptr[c1];
+            }
+        };
+        int64_t rs_n, re_n;
+        bounds(first, rs_n, re_n);
+        for (int64_t t = first; t < ntiles; t += step, ++k) {
+            const int st = (int)(k % kGapStages);
+            const int64_t rs = rs_n, re = re_n;
+            bounds(t + step, rs_n, re_n);
+            if (k >= kGapStages) {
+                if (!gap_wait(smem_u32(&sm.empty[st]), (uint32_t)((k / kGapStages) - 1) & 1u, abort_flag, status)) break;
+            }
+            if (lane == 0) {
+                const int64_t w0 = rs & ~(int64_t)3;
+                const int64_t elems = ((re - w0) + 3) & ~(int64_t)3;
+                const uint32_t bar = smem_u32(&sm.full[st]);
+                // the stage was read by ordinary loads: order them before the copy engine's writes
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                if (elems > 0 && elems <= kGapStageElems) {
+                    sm.base[st] = w0;
+                    const uint32_t bytes = (uint32_t)elems * 4u;
+                    mbar_arrive_expect_tx(bar, 2u * bytes);
+                    bulk_g2s(smem_u32(&sm.idx[st][0]), indices + w0, bytes, bar);
+                    bulk_g2s(smem_u32(&sm.val[st][0]), values + w0, bytes, bar);
+                } else {
+                    sm.base[st] = -1; // empty tile, or too many non-zeros for a stage: the consumers read global memory
+                    __threadfence_block();
+                    mbar_arrive(bar);
+                }
+            }
+            __syncwarp();
+        }
+    } else {
+        // ------------------------------------------------ consumers
+        const int r = tid / TPR, sub = tid % TPR;
+        int64_t k = 0;
+        // the extent and the scalars of this thread's coordinate in the next tile are fetched a tile ahead
+        auto fetch = [&](int64_t t, int64_t &rs, int64_t &re, float &lab, float &sta) {
+            rs = re = 0;
+            lab = sta = 0.0f;
+            const int64_t c = t * R + r;
+            if (t < ntiles && c < n_coord) {
+                rs = indptr[c];
+                re = indptr[c + 1];
+                sta = state[c];
+                if (LOSS != CHICLE_LOSS_RIDGE_PRIMAL) lab = labels[c];
+            }
+        };
+        int64_t rs_n, re_n;
+        float lab_n, sta_n;
+        fetch(first, rs_n, re_n, lab_n, sta_n);
+        for (int64_t t = first; t < ntiles; t += step, ++k) {
+            const int st = (int)(k % kGapStages);
+            const int64_t rs = rs_n, re = re_n;
+            const float lab = lab_n, sta = sta_n;
+            const bool owner = sub == 0 && t * R + r < n_coord;
+            fetch(t + step, rs_n, re_n, lab_n, sta_n);
+            if (!gap_wait(smem_u32(&sm.full[st]), (uint32_t)(k / kGapStages) & 1u, abort_flag, status)) break;
+            const int64_t base = sm.base[st];
+            double dot = 0.0;
+            for (int64_t e0 = rs + sub; e0 < re; e0 += (int64_t)TPR * kMaxPer) {
+                int32_t ii[kMaxPer];
+                float xx[kMaxPer], tt[kMaxPer], yy[kMaxPer], hh[kMaxPer];
+#pragma unroll
+                for (int q = 0; q < kMaxPer; ++q) {
+                    const int64_t e = e0 + (int64_t)q * TPR;
+                    ii[q] = -1;
+                    xx[q] = 0.0f;
+                    if (e < re) {
+                        if (base >= 0) {
+                            ii[q] = sm.idx[st][e - base];
+                            xx[q] = sm.val[st][e - base];
+                        } else {
+                            ii[q] = indices[e];
+                            xx[q] = values[e];
+                        }
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < kMaxPer; ++q) {
+                    const bool far = ii[q] >= hot_n;
+                    hh[q] = sm.vhot[(ii[q] >= 0 && !far) ? ii[q] : 0];
+                    tt[q] = far ? vec[ii[q]] : 0.0f;
+                    yy[q] = (LOSS == CHICLE_LOSS_RIDGE_PRIMAL && far) ? labels[ii[q]] : 0.0f;
+                }
+#pragma unroll
+                for (int q = 0; q < kMaxPer; ++q) {
+                    // (x is 0 beyond the coordinate's end; fp32 v - y for the staged head, as the solvers' residual)
+                    const double t = ii[q] >= hot_n ? (double)tt[q] - (double)yy[q] : (double)hh[q];
+                    dot = fma((double)xx[q], t, dot);
+                }
+            }
+            // the stage is free once every lane of the warp has read its entries
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm.empty[st]));
+#pragma unroll
+            for (int o = 1; o < TPR; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            if (owner) gap_term<LOSS>(dot, lab, sta, inv_lam_n, s0, s1);
+        }
+    }
+    // slice of the shared vector owned by this block (consumer threads)
+    double s2 = 0.0, s3 = 0.0;
+    if (tid < kGapConsumers) {
+        const int64_t chunk = (dim + gridDim.x - 1) / gridDim.x;
+        const int64_t b = (int64_t)blockIdx.x * chunk;
+        const int64_t e = b + chunk < dim ? b + chunk : dim;
+        for (int64_t j = b + tid; j < e; j += kGapConsumers) {
+            if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+                const double y = (double)labels[j]; // targets
+                const double rr = (double)vec[j] - y;
+                s2 = fma(rr, rr, s2);
+                s3 = fma(rr, y, s3);
+            } else {
+                const double t = (double)vec[j];
+                s2 = fma(t, t, s2);
+            }
+        }
+        s2 = warp_sum_d(s2);
+        s3 = warp_sum_d(s3);
+        sm.sh[tid][0] = s0;
+        sm.sh[tid][1] = s1;
+        if (lane == 0) {
+            sm.sh2[warp][0] = s2;
+            sm.sh2[warp][1] = s3;
+        }
+    }
+    __syncthreads();
+    // fixed-order combination: threads in index order for the per-coordinate sums, warps in order for the slices
+    if (tid < 2) {
+        double tot = 0.0;
+        for (int w = 0; w < kGapConsumers / 32; ++w) {
+            double a = 0.0;
+            for (int l = 0; l < 32; ++l) a += sm.sh[w * 32 + l][tid];
+            tot += a;
+        }
+        partials[(size_t)blockIdx.x * 4 + tid] = tot;
+    } else if (tid < 4) {
+        double tot = 0.0;
+        for (int w = 0; w < kGapConsumers / 32; ++w) tot += sm.sh2[w][tid - 2];
+        partials[(size_t)blockIdx.x * 4 + tid] = tot;
     }
 }
 
@@ -425,31 +655,48 @@ cudaError_t launch_refresh_resid(Glm &g)
     return cudaGetLastError();
 }
 
-cudaError_t launch_gap(Glm &g)
+template <int LOSS, int R> cudaError_t launch_gap_stream(Glm &g, int nb, double lam_n)
 {
-    const int nb = g.gap_blocks;
+    auto kern = k_gap_stream<LOSS, R>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(GapShared));
+    if (e != cudaSuccess) return e;
+    kern<<<nb, kGapConsumers + 32, sizeof(GapShared), g.stream>>>(g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.n_coord,
+                                                                   g.dim, lam_n, g.gap_partials, g.d_status);
+    return cudaGetLastError();
+}
+
+template <int LOSS> cudaError_t launch_gap_loss(Glm &g)
+{
     const double n = (double)g.n_examples;
     const double lam_n = (double)g.lambda * n;
-    switch (g.loss) {
-    case CHICLE_LOSS_HINGE_DUAL:
-        k_gap_partials<CHICLE_LOSS_HINGE_DUAL><<<nb, kThreads, 0, g.stream>>>(
-            g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord, g.dim, lam_n, g.gap_partials);
-        k_gap_final<CHICLE_LOSS_HINGE_DUAL><<<1, 128, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda, g.gap_out);
-        break;
-    case CHICLE_LOSS_LOGISTIC_DUAL:
-        k_gap_partials<CHICLE_LOSS_LOGISTIC_DUAL><<<nb, kThreads, 0, g.stream>>>(
-            g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord, g.dim, lam_n, g.gap_partials);
-        k_gap_final<CHICLE_LOSS_LOGISTIC_DUAL><<<1, 128, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda,
-                                                                        g.gap_out);
-        break;
-    default:
-        k_gap_partials<CHICLE_LOSS_RIDGE_PRIMAL><<<nb, kThreads, 0, g.stream>>>(
-            g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord, g.dim, lam_n, g.gap_partials);
-        k_gap_final<CHICLE_LOSS_RIDGE_PRIMAL><<<1, 128, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda,
-                                                                       g.gap_out);
-        break;
+    int nb = g.gap_blocks;
+    const char *force = getenv("CHICLE_FORCE_VARIANT"); // debugging aid: "gapwarp" selects the warp-per-coordinate kernel
+    if (g.indptr && g.hot_variant && !(force && strcmp(force, "gapwarp") == 0)) {
+        // skewed ids: the streamed kernel, one block per SM; coordinates per tile: as many as keep a tile's non-zeros
+        // comfortably inside a stage
+        nb = g.sm_count < g.gap_blocks ? g.sm_count : g.gap_blocks;
+        const double avg = (double)g.nnz / (double)g.n_coord;
+        cudaError_t e;
+        if (avg * 128 <= 3300) e = launch_gap_stream<LOSS, 128>(g, nb, lam_n);
+        else if (avg * 64 <= 3300) e = launch_gap_stream<LOSS, 64>(g, nb, lam_n);
+        else if (avg * 32 <= 3300) e = launch_gap_stream<LOSS, 32>(g, nb, lam_n);
+        else e = launch_gap_stream<LOSS, 16>(g, nb, lam_n);
+        if (e != cudaSuccess) return e;
+    } else {
+        k_gap_partials<LOSS><<<nb, kThreads, 0, g.stream>>>(g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord,
+                                                            g.dim, lam_n, g.gap_partials);
     }
+    k_gap_final<LOSS><<<1, 128, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda, g.gap_out);
     return cudaGetLastError();
+}
+
+cudaError_t launch_gap(Glm &g)
+{
+    switch (g.loss) {
+    case CHICLE_LOSS_HINGE_DUAL: return launch_gap_loss<CHICLE_LOSS_HINGE_DUAL>(g);
+    case CHICLE_LOSS_LOGISTIC_DUAL: return launch_gap_loss<CHICLE_LOSS_LOGISTIC_DUAL>(g);
+    default: return launch_gap_loss<CHICLE_LOSS_RIDGE_PRIMAL>(g);
+    }
 }
 
 cudaError_t launch_shared_vector(Glm &g)
