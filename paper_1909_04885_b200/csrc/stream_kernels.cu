@@ -361,6 +361,14 @@ __device__ __forceinline__ bool gap_wait(uint32_t bar, uint32_t parity, volatile
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
+__device__ __forceinline__ float gap_ldg_if(const float *p, bool on)
+{
+    float v;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\tmov.f32 %0, 0f00000000;\n\t@q ld.global.nc.f32 %0, [%1];\n\t}"
+                 : "=f"(v) : "l"(p), "r"((uint32_t)on));
+    return v;
+}
+
 struct GapShared {
     alignas(16) float vhot[kGapHot];       // the head of the shared vector (ridge: of v - y)
     alignas(16) int32_t idx[kGapStages][kGapStageElems];
@@ -469,36 +477,45 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
             if (!gap_wait(smem_u32(&sm.full[st]), (uint32_t)(k / kGapStages) & 1u, abort_flag, status)) break;
             const int64_t base = sm.base[st];
             double dot = 0.0;
-            for (int64_t e0 = rs + sub; e0 < re; e0 += (int64_t)TPR * kMaxPer) {
-                int32_t ii[kMaxPer];
-                float xx[kMaxPer], tt[kMaxPer], yy[kMaxPer], hh[kMaxPer];
+            if (base >= 0) {
+                // staged: 32-bit offsets into the stage, every load unconditional (clamped) and the gathers beyond the
+                // staged head of the vector predicated, so that nothing branches per non-zero
+                const int hi = (int)(re - base);
+                const uint32_t a_idx = smem_u32(&sm.idx[st][0]), a_val = smem_u32(&sm.val[st][0]);
+                for (int e0 = (int)(rs - base) + sub; e0 < hi; e0 += TPR * kMaxPer) {
+                    int32_t ii[kMaxPer];
+                    float xx[kMaxPer], tt[kMaxPer], yy[kMaxPer], hh[kMaxPer];
 #pragma unroll
-                for (int q = 0; q < kMaxPer; ++q) {
-                    const int64_t e = e0 + (int64_t)q * TPR;
-                    ii[q] = -1;
-                    xx[q] = 0.0f;
-                    if (e < re) {
-                        if (base >= 0) {
-                            ii[q] = sm.idx[st][e - base];
-                            xx[q] = sm.val[st][e - base];
-                        } else {
-                            ii[q] = indices[e];
-                            xx[q] = values[e];
-                        }
+                    for (int q = 0; q < kMaxPer; ++q) {
+                        const int e = e0 + q * TPR;
+                        const bool valid = e < hi;
+                        const uint32_t o = 4u * (uint32_t)(valid ? e : 0);
+                        const int32_t i = lds_s32(a_idx + o);
+                        const float x = lds_f32(a_val + o);
+                        ii[q] = valid ? i : 0;
+                        xx[q] = valid ? x : 0.0f;
+                    }
+#pragma unroll
+                    for (int q = 0; q < kMaxPer; ++q) {
+                        const bool far = ii[q] >= hot_n;
+                        hh[q] = sm.vhot[far ? 0 : ii[q]];
+                        tt[q] = gap_ldg_if(vec + (far ? ii[q] : 0), far);
+                        yy[q] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? gap_ldg_if(labels + (far ? ii[q] : 0), far) : 0.0f;
+                    }
+#pragma unroll
+                    for (int q = 0; q < kMaxPer; ++q) {
+                        // (x is 0 beyond the coordinate's end; fp32 v - y for the staged head, as the solvers' residual)
+                        const double t = ii[q] >= hot_n ? (double)tt[q] - (double)yy[q] : (double)hh[q];
+                        dot = fma((double)xx[q], t, dot);
                     }
                 }
-#pragma unroll
-                for (int q = 0; q < kMaxPer; ++q) {
-                    const bool far = ii[q] >= hot_n;
-                    hh[q] = sm.vhot[(ii[q] >= 0 && !far) ? ii[q] : 0];
-                    tt[q] = far ? vec[ii[q]] : 0.0f;
-                    yy[q] = (LOSS == CHICLE_LOSS_RIDGE_PRIMAL && far) ? labels[ii[q]] : 0.0f;
-                }
-#pragma unroll
-                for (int q = 0; q < kMaxPer; ++q) {
-                    // (x is 0 beyond the coordinate's end; fp32 v - y for the staged head, as the solvers' residual)
-                    const double t = ii[q] >= hot_n ? (double)tt[q] - (double)yy[q] : (double)hh[q];
-                    dot = fma((double)xx[q], t, dot);
+            } else {
+                for (int64_t e = rs + sub; e < re; e += TPR) {
+                    const int32_t i = indices[e];
+                    double t;
+                    if (i < hot_n) t = (double)sm.vhot[i];
+                    else t = (double)vec[i] - (LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? (double)labels[i] : 0.0);
+                    dot = fma((double)values[e], t, dot);
                 }
             }
             // the stage is free once every lane of the warp has read its entries
