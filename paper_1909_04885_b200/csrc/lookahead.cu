@@ -31,8 +31,8 @@
 // bulk copies each slowed whatever phase ran while those 64 copies landed by about 3 000 cycles per block (the
 // slow phase moved with the point of issue), three times what the recurrence itself costs.
 //
-// Blocks the shared-memory buffers cannot hold (a coordinate longer than 128 entries, more distinct ids than TMAX)
-// are flagged by the prepare kernel and walked coordinate by coordinate by warp 0. Rounds that span several local
+// A block with a coordinate longer than 128 entries does not fit the shared-memory buffers: the prepare kernel
+// flags it and warp 0 walks it coordinate by coordinate. Rounds that span several local
 // epochs revisit coordinates, whose state the headers would not know: those take the blocked solver instead.
 #include <cstdio>
 #include <cstdlib>

@@ -215,7 +215,7 @@ def test_lookahead_solver_is_the_default_for_single_epoch_rounds():
 
 
 def test_lookahead_blocks_that_do_not_fit_are_walked_in_place():
-    # rows longer than a staged row (128 entries) and a block with more distinct ids than the buffers hold
+    # rows longer than a staged row (128 entries), and blocks of long rows with hardly any id in common
     run_parity(tiny_csr(200, 3000, seed=9, K=2, density=0.03, long_row=500))
     rng = np.random.default_rng(4)
     n, d = 256, 40000
