@@ -381,14 +381,14 @@ struct GapShared {
     int abort_flag;
 };
 
-template <int LOSS, int R>
+template <int LOSS, int R, int PER>
 __global__ void __launch_bounds__(kGapConsumers + 32, 1)
 k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices, const float *__restrict__ values,
              const float *__restrict__ labels, const float *__restrict__ state, const float *__restrict__ vec,
              int64_t n_coord, int64_t dim, double lam_n, double *__restrict__ partials, uint32_t *status)
 {
     constexpr int TPR = kGapConsumers / R; // threads per coordinate
-    constexpr int kMaxPer = 8;             // entries a thread keeps in flight
+    constexpr int kMaxPer = PER;           // entries a thread keeps in flight (6 or 8: the fewer idle slots, the fewer instructions)
     extern __shared__ __align__(128) unsigned char gap_smem[];
     GapShared &sm = *reinterpret_cast<GapShared *>(gap_smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -490,9 +490,8 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
                         const int e = e0 + q * TPR;
                         const bool valid = e < hi;
                         const uint32_t o = 4u * (uint32_t)(valid ? e : 0);
-                        const int32_t i = lds_s32(a_idx + o);
+                        ii[q] = lds_s32(a_idx + o); // (a slot beyond the coordinate's end reads the stage's first entry with x = 0)
                         const float x = lds_f32(a_val + o);
-                        ii[q] = valid ? i : 0;
                         xx[q] = valid ? x : 0.0f;
                     }
 #pragma unroll
@@ -505,8 +504,12 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
 #pragma unroll
                     for (int q = 0; q < kMaxPer; ++q) {
                         // (x is 0 beyond the coordinate's end; fp32 v - y for the staged head, as the solvers' residual)
-                        const double t = ii[q] >= hot_n ? (double)tt[q] - (double)yy[q] : (double)hh[q];
-                        dot = fma((double)xx[q], t, dot);
+                        if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
+                            const double t = ii[q] >= hot_n ? (double)tt[q] - (double)yy[q] : (double)hh[q];
+                            dot = fma((double)xx[q], t, dot);
+                        } else {
+                            dot = fma((double)xx[q], (double)(ii[q] >= hot_n ? tt[q] : hh[q]), dot);
+                        }
                     }
                 }
             } else {
@@ -672,14 +675,22 @@ cudaError_t launch_refresh_resid(Glm &g)
     return cudaGetLastError();
 }
 
-template <int LOSS, int R> cudaError_t launch_gap_stream(Glm &g, int nb, double lam_n)
+template <int LOSS, int R, int PER> cudaError_t launch_gap_stream_per(Glm &g, int nb, double lam_n)
 {
-    auto kern = k_gap_stream<LOSS, R>;
+    auto kern = k_gap_stream<LOSS, R, PER>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(GapShared));
     if (e != cudaSuccess) return e;
     kern<<<nb, kGapConsumers + 32, sizeof(GapShared), g.stream>>>(g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.n_coord,
                                                                    g.dim, lam_n, g.gap_partials, g.d_status);
     return cudaGetLastError();
+}
+
+template <int LOSS, int R> cudaError_t launch_gap_stream(Glm &g, int nb, double lam_n)
+{
+    // entries a thread keeps in flight: 6 where that covers the average coordinate with some room, else 8
+    const double avg = (double)g.nnz / (double)g.n_coord;
+    if (avg * 1.15 <= 6.0 * (kGapConsumers / R)) return launch_gap_stream_per<LOSS, R, 6>(g, nb, lam_n);
+    return launch_gap_stream_per<LOSS, R, 8>(g, nb, lam_n);
 }
 
 template <int LOSS> cudaError_t launch_gap_loss(Glm &g)
