@@ -60,7 +60,7 @@ struct alignas(16) LookHdr {
     int32_t nnz;
     float p0, p1, p2, p3; // the constants of the scalar step (see coordinate_step)
     float q0;             // what the states of the block's earlier coordinates at round start contribute (see below)
-    float pad[3];
+    float pad[3];         // [0]: log of p2 for the logistic loss (the start of its Newton iteration needs it)
 };
 static_assert(sizeof(LookHdr) == 48, "header size");
 
@@ -148,7 +148,10 @@ template <int LOSS> __device__ __forceinline__ LookHdr make_hdr(const SolverPara
         hd.p1 = y * al;
         hd.p3 = y;
         if (LOSS == CHICLE_LOSS_HINGE_DUAL) hd.p2 = s > 0.0f ? P.lam_n / (P.sigma * s) : CUDART_INF_F;
-        else hd.p2 = P.sigma * s / P.lam_n;
+        else {
+            hd.p2 = P.sigma * s / P.lam_n;
+            hd.pad[0] = hd.p2 > 0.0f ? logf(hd.p2) : -CUDART_INF_F; // log q, for the start of the Newton iteration
+        }
     }
     return hd;
 }
@@ -199,7 +202,7 @@ template <int LOSS> __device__ __forceinline__ float recurrence_map(float s, con
 {
     if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) return -s * h.p2;
     if (LOSS == CHICLE_LOSS_HINGE_DUAL) return __saturatef(s);
-    return logistic_root(s, h.p2);
+    return logistic_root(s, h.p2, h.pad[0]);
 }
 
 __device__ __forceinline__ uint32_t hash_id(int32_t id) { return ((uint32_t)id * 2654435761u) >> 20; } // 12 bits

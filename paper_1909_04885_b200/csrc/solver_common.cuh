@@ -190,24 +190,29 @@ __device__ __forceinline__ float warp_sum(float x)
 
 // a' = sigmoid(z) at the root of z + q sigmoid(z) = c: the root is taken on the convex branch z <= 0 (a positive root
 // is reflected first), Newton from a Lambert-W-like start, fixed iteration count.
-__device__ __forceinline__ float logistic_root(float c, float q)
+// `log_q` is log(q) (-inf for q = 0): a constant of the coordinate, so callers that prepare their constants ahead pass it.
+__device__ __forceinline__ float logistic_root(float c, float q, float log_q)
 {
     const bool flip = c > 0.5f * q;
     if (flip) c = q - c;
-    const float kappa = q > 0.0f ? __logf(q) + c : -CUDART_INF_F;
+    const float kappa = log_q + c;
     float z = kappa <= 0.0f ? fminf(c, 0.0f) : fminf(c - (kappa - __logf(1.0f + kappa)), 0.0f);
 #pragma unroll
     for (int it = 0; it < kNewtonIters; ++it) {
+        // the Newton step F / F' with F = z + q p - c, F' = 1 + q p (1 - p), p = e / (1 + e), brought to one
+        // denominator: ((z - c) s^2 + q e s) / (s^2 + q e), s = 1 + e: one exponential and one division per step
         const float e = __expf(z);
-        const float r = __frcp_rn(1.0f + e);
-        const float p = e * r;
-        const float F = fmaf(q, p, z) - c;
-        const float Fp = fmaf(q * p, r, 1.0f); // 1 + q p (1 - p), 1 - p = 1 / (1 + e)
-        z = fminf(z - __fdividef(F, Fp), 0.0f);
+        const float s = 1.0f + e, s2 = s * s, qe = q * e;
+        z = fminf(z - __fdividef(fmaf(z - c, s2, qe * s), s2 + qe), 0.0f);
     }
     const float e = __expf(z);
     const float r = __frcp_rn(1.0f + e);
     return flip ? r : e * r;
+}
+
+__device__ __forceinline__ float logistic_root(float c, float q)
+{
+    return logistic_root(c, q, q > 0.0f ? __logf(q) : -CUDART_INF_F);
 }
 
 // Scalar steps. `dot` is x_c . v_local (dual) or c_j . (v_local - y) (ridge). Returns delta and the new state.
