@@ -226,6 +226,25 @@ def test_lookahead_blocks_that_do_not_fit_are_walked_in_place():
     run_parity(Workload("wide_blocks", "hinge", "csr", n, d, vals, y, 1.0 / n, 3, [Phase(0, 2, 0, 2.0)], indptr, idx))
 
 
+def test_gap_tile_that_does_not_fit_a_stage_is_read_in_place():
+    # many short rows (so that the streamed gap kernel takes 128 coordinates per tile) and two neighbouring rows of
+    # 3 000 entries each: their tile has more non-zeros than a stage of the ring holds; some empty rows as well
+    rng = np.random.default_rng(21)
+    n, d = 1500, 4000
+    X = rng.standard_normal((n, d)).astype(np.float32) * 0.1
+    X[rng.random((n, d)) > 0.005] = 0.0
+    for r in (700, 701):
+        X[r, :3000] = rng.standard_normal(3000).astype(np.float32) * 0.02 + 0.01
+    X[10:14] = 0.0
+    w = rng.standard_normal(d)
+    y = np.where(X @ w >= 0, 1.0, -1.0).astype(np.float32)
+    indptr = np.zeros(n + 1, np.int64)
+    indptr[1:] = np.cumsum((X != 0).sum(1))
+    wl = Workload("gap_overflow", "hinge", "csr", n, d, X[X != 0].astype(np.float32), y, 1.0 / n, 3, [Phase(0, 4, 0, 4.0)],
+                  indptr, np.nonzero(X)[1].astype(np.int32))
+    run_parity(wl)
+
+
 def test_lookahead_runs_are_bit_reproducible():
     w = datagen.make("hinge_csr", 100)
     res = []
