@@ -216,29 +216,31 @@ __device__ __forceinline__ bool take_record(const LookParams &P, uint32_t bytes,
 }
 
 // ------------------------------------------------------------------------------------------------ prepare
-struct PreShared {
-    int32_t idx[kMaxNz];     // the block's non-zeros, row after row
-    float val[kMaxNz];
-    uint16_t slot[kMaxNz];   // table slot of each non-zero's id
-    int32_t key[kHT];        // id in a table slot, -1 = empty
-    uint32_t mask[kHT];      // bit j: coordinate j of the block has this id
-    uint16_t soff[kHT];      // start of the slot's list
-    float lval[kMaxNz];      // the values of the non-zeros with shared ids, list after list (for the Gram pass)
+template <int NZ, int HT, int THREADS> struct PreShared {
+    int32_t idx[NZ];     // the block's non-zeros, row after row
+    float val[NZ];
+    uint16_t slot[NZ];   // table slot of each non-zero's id
+    int32_t key[HT];        // id in a table slot, -1 = empty
+    uint32_t mask[HT];      // bit j: coordinate j of the block has this id
+    uint16_t soff[HT];      // start of the slot's list
+    float lval[NZ];      // the values of the non-zeros with shared ids, list after list (for the Gram pass)
     float G[kLB][kLB + 1];
     int64_t rs[kLB];
     int32_t nnz[kLB];
     int32_t roff[kLB + 1];
-    uint32_t warp_tot[kPreThreadsS / 32];
+    uint32_t warp_tot[THREADS / 32];
     float gsc[kLB], ys[kLB], as[kLB]; // per coordinate: its Gram scale, and what multiplies / enters from the earlier ones
     int32_t total, too_long;
     uint32_t bytes;
     unsigned long long offset;
 };
 
-template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahead_prepare(const LookParams P)
+template <int LOSS, int NZ, int HT, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) k_lookahead_prepare(const LookParams P)
 {
     extern __shared__ __align__(16) unsigned char smem_pre[];
-    PreShared &sh = *reinterpret_cast<PreShared *>(smem_pre);
+    using Shared = PreShared<NZ, HT, THREADS>;
+    Shared &sh = *reinterpret_cast<Shared *>(smem_pre);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t bid = blockIdx.x;
     int k;
@@ -275,14 +277,16 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
             const int t = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += t;
         }
-        sh.roff[lane] = too_long ? 0 : incl - hd.nnz;
+        // (a block with more non-zeros than this variant's arrays hold is walked in place as well)
+        const bool over = too_long || __shfl_sync(0xffffffffu, incl, 31) > NZ;
+        sh.roff[lane] = over ? 0 : incl - hd.nnz;
         if (lane == 31) {
-            sh.roff[kLB] = incl;
-            sh.total = incl;
-            sh.too_long = too_long ? 1 : 0;
+            sh.roff[kLB] = over ? 0 : incl;
+            sh.total = over ? 0 : incl;
+            sh.too_long = over ? 1 : 0;
         }
     }
-    for (int p = tid; p < kHT; p += kPreThreadsS) {
+    for (int p = tid; p < HT; p += THREADS) {
         sh.key[p] = -1;
         sh.mask[p] = 0u;
     }
@@ -292,7 +296,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     bool slow = sh.too_long != 0;
     if (!slow) {
         // ---- the block's non-zeros into shared memory, every id into the table
-        for (int j = warp; j < cnt; j += kPreThreadsS / 32) {
+        for (int j = warp; j < cnt; j += THREADS / 32) {
             const int n = sh.nnz[j], r0 = sh.roff[j];
             const int64_t rs = sh.rs[j];
             int32_t ids4[kCapL / 32];
@@ -310,15 +314,15 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
                 const int32_t id = ids4[c];
                 sh.idx[r0 + e] = id;
                 sh.val[r0 + e] = vals4[c];
-                uint32_t p = hash_id(id);
-                for (int probe = 0; probe < kHT; ++probe) {
+                uint32_t p = hash_id(id) & (HT - 1);
+                for (int probe = 0; probe < HT; ++probe) {
                     int32_t seen = sh.key[p];
                     if (seen == -1) {
                         seen = atomicCAS(&sh.key[p], -1, id);
                         if (seen == -1) break;
                     }
                     if (seen == id) break;
-                    p = (p + 1) & (kHT - 1);
+                    p = (p + 1) & (HT - 1);
                 }
                 atomicOr(&sh.mask[p], 1u << j);
                 sh.slot[r0 + e] = (uint16_t)p;
@@ -332,7 +336,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     //      of the threads before it
     uint32_t mine = 0;
     if (!slow)
-        for (int p = tid; p < kHT; p += kPreThreadsS) {
+        for (int p = tid; p < HT; p += THREADS) {
             const uint32_t m = sh.mask[p];
             if (m & (m - 1u)) mine += (1u << 16) + (uint32_t)__popc(m);
         }
@@ -346,7 +350,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     __syncthreads();
     PRE_T(2);
     uint32_t run = incl - mine, all = 0;
-    for (int w2 = 0; w2 < kPreThreadsS / 32; ++w2) {
+    for (int w2 = 0; w2 < THREADS / 32; ++w2) {
         if (w2 < warp) run += sh.warp_tot[w2];
         all += sh.warp_tot[w2];
     }
@@ -383,7 +387,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     int32_t *ids_g = idx_g + total;
     uint16_t *cpos_g = reinterpret_cast<uint16_t *>(ids_g + T);
     uint16_t *off_g = cpos_g + total;
-    for (int p = tid; p < kHT; p += kPreThreadsS) {
+    for (int p = tid; p < HT; p += THREADS) {
         const uint32_t m = sh.mask[p];
         if (m & (m - 1u)) {
             const uint32_t t = run >> 16, o = run & 0xffffu;
@@ -397,7 +401,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     __syncthreads();
     PRE_T(4);
     // ---- list entries: a non-zero's place in its id's list is the number of lower coordinates that have the id
-    for (int j = warp; j < cnt; j += kPreThreadsS / 32) {
+    for (int j = warp; j < cnt; j += THREADS / 32) {
         const int n = sh.nnz[j], r0 = sh.roff[j];
         for (int e = lane; e < n; e += 32) {
             const int p = sh.slot[r0 + e];
@@ -421,7 +425,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     // ---- Gram triangle: a warp per coordinate j, lane l collects x_j . x_l over j's entries in ascending order. The
     //      lanes first look at 32 entries at once and keep those whose id an earlier coordinate has too; only these
     //      are then walked, their mask, list start and value handed round by shuffles.
-    for (int j = warp; j < kLB; j += kPreThreadsS / 32) {
+    for (int j = warp; j < kLB; j += THREADS / 32) {
         float acc = 0.0f;
         if (j < cnt) {
             const int n = sh.nnz[j], r0 = sh.roff[j];
@@ -465,7 +469,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreadsS, 2) k_lookahe
     }
     __syncthreads();
     PRE_T(6);
-    for (int i = tid; i < kLB * kLB; i += kPreThreadsS) out.G[i] = sh.G[i >> 5][i & 31];
+    for (int i = tid; i < kLB * kLB; i += THREADS) out.G[i] = sh.G[i >> 5][i & 31];
     PRE_T(7);
 }
 
@@ -978,6 +982,16 @@ template <int LOSS, bool DENSE, int HOT, int TMAX, int NCH> cudaError_t launch_c
     return e;
 }
 
+template <int LOSS, int NZ, int HT, int THREADS> cudaError_t launch_prepare(Glm &g, const LookParams &P, unsigned nb)
+{
+    using Shared = PreShared<NZ, HT, THREADS>;
+    auto pre = k_lookahead_prepare<LOSS, NZ, HT, THREADS>;
+    cudaError_t e = cudaFuncSetAttribute(pre, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Shared));
+    if (e != cudaSuccess) return e;
+    pre<<<nb, THREADS, sizeof(Shared), g.stream>>>(P);
+    return cudaGetLastError();
+}
+
 template <int LOSS> cudaError_t launch_loss(Glm &g, LookParams &P)
 {
     const unsigned nb = (unsigned)P.n_blocks;
@@ -990,11 +1004,10 @@ template <int LOSS> cudaError_t launch_loss(Glm &g, LookParams &P)
         if (g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
         return launch_chain<LOSS, true, kCapL, 4, 4>(g, P);
     }
-    auto pre = k_lookahead_prepare<LOSS>;
-    e = cudaFuncSetAttribute(pre, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PreShared));
-    if (e != cudaSuccess) return e;
-    pre<<<nb, kPreThreadsS, sizeof(PreShared), g.stream>>>(P);
-    e = cudaGetLastError();
+    // blocks of up to 2 048 non-zeros (32 coordinates of 50 on average, with room): the small variant, four CTAs per SM
+    const double avg_block = 32.0 * (double)g.nnz / (double)g.n_coord;
+    if (avg_block * 1.25 <= 2048.0) e = launch_prepare<LOSS, 2048, 2048, 256>(g, P, nb);
+    else e = launch_prepare<LOSS, kMaxNz, kHT, kPreThreadsS>(g, P, nb);
     if (e != cudaSuccess) return e;
 #ifdef CHICLE_LA_TIMING
     {
