@@ -325,7 +325,7 @@ def run_b200(args):
     prep_bytes = comp_bytes + w.nnz * 16 + (w.n_coord // 32) * 5728
     traffic = read_traffic() if args.scale == 1 else None
     owner_passes = 1 if ph.K <= 256 else 2
-    launches = 1 + 5 * (8 + owner_passes) + 2 + 1 + 2   # order keys + radix passes, solver (2), aggregation, gap (2)
+    launches = 1 + 5 * (4 + owner_passes) + 1 + 2 + 1 + 2   # order keys, radix passes, run fix-up, solver (2), aggregation, gap (2)
 
     cpu_baseline = time_oracle(w, ph, args.cpu_rounds) if args.cpu_rounds >= 0 else None
 

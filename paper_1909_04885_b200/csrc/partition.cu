@@ -94,6 +94,32 @@ cudaError_t launch_partition(Glm &g, int32_t K, uint64_t seed)
     return cudaGetLastError();
 }
 
+// After a stable sort on the upper 32 key bits only: elements whose upper halves agree stand next to each other in
+// their old order; the thread at the head of such a run (they are rare and short: keys are 64-bit hashes) puts it
+// into full-key order by insertion. Runs are disjoint, so the threads do not meet.
+__global__ void k_order_runs(int64_t n, uint64_t *__restrict__ keys, int32_t *__restrict__ vals)
+{
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i + 1 < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint32_t hi = (uint32_t)(keys[i] >> 32);
+        if ((uint32_t)(keys[i + 1] >> 32) != hi) continue;
+        if (i > 0 && (uint32_t)(keys[i - 1] >> 32) == hi) continue; // not the head of the run
+        int64_t end = i + 2;
+        while (end < n && (uint32_t)(keys[end] >> 32) == hi) ++end;
+        for (int64_t a = i + 1; a < end; ++a) {
+            const uint64_t ka = keys[a];
+            const int32_t va = vals[a];
+            int64_t b = a;
+            while (b > i && keys[b - 1] > ka) {
+                keys[b] = keys[b - 1];
+                vals[b] = vals[b - 1];
+                --b;
+            }
+            keys[b] = ka;
+            vals[b] = va;
+        }
+    }
+}
+
 cudaError_t launch_permutation(Glm &g, int64_t round, int64_t epochs)
 {
     const int64_t n = g.n_coord;
@@ -103,12 +129,19 @@ cudaError_t launch_permutation(Glm &g, int64_t round, int64_t epochs)
     for (int64_t e = 0; e < epochs; ++e) {
         const uint64_t b = mix64(((uint64_t)round << 32) + (uint64_t)e);
         k_perm_keys<<<blocks_for(n, T), T, 0, g.stream>>>(n, a ^ b, g.members, w.keys[0], w.vals[0]);
+        // four radix passes over the upper half of the 64-bit keys, then the rare runs with equal upper halves are
+        // put into full-key order: the same order as eight passes give, at half the passes
         int cur = 0;
-        for (int pass = 0; pass < 8; ++pass) {
+        for (int pass = 4; pass < 8; ++pass) {
             cudaError_t err = radix_pass(w.keys[cur], w.vals[cur], w.keys[cur ^ 1], w.vals[cur ^ 1], nullptr, n,
                                          8 * pass, w.hist, w.scan_sums, g.stream);
             if (err != cudaSuccess) return err;
             cur ^= 1;
+        }
+        {
+            unsigned grid = blocks_for(n, T);
+            if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
+            k_order_runs<<<grid, T, 0, g.stream>>>(n, w.keys[cur], w.vals[cur]);
         }
         cudaError_t err = owner_passes(g, g.K, w.vals[cur], reinterpret_cast<int32_t *>(w.keys[0]),
                                        g.perm + (size_t)e * (size_t)n);
