@@ -71,29 +71,6 @@ cudaError_t owner_passes(Glm &g, int32_t K, const int32_t *in, int32_t *scratch,
 
 } // namespace
 
-cudaError_t launch_partition(Glm &g, int32_t K, uint64_t seed)
-{
-    const int64_t n = g.n_coord;
-    SortWorkspace &w = g.sortws;
-    const int T = 256;
-    k_partition_keys<<<blocks_for(n, T), T, 0, g.stream>>>(n, mix64(seed), w.keys[0], w.vals[0]);
-    int cur = 0;
-    for (int pass = 0; pass < 8; ++pass) {
-        cudaError_t e = radix_pass(w.keys[cur], w.vals[cur], w.keys[cur ^ 1], w.vals[cur ^ 1], nullptr, n, 8 * pass,
-                                   w.hist, w.scan_sums, g.stream);
-        if (e != cudaSuccess) return e;
-        cur ^= 1;
-    }
-    // 8 passes: the sorted ids are back in buffer 0
-    k_owner_from_rank<<<blocks_for(n, T), T, 0, g.stream>>>(n, n / K, n % K, w.vals[cur], g.owner);
-    // members: ids 0..n-1 (ascending) stably grouped by owner
-    k_iota<<<blocks_for(n, T), T, 0, g.stream>>>(n, w.vals[0]);
-    // in = vals[0]; scratch = reinterpret keys[0] storage as int32 (keys are dead now)
-    cudaError_t e = owner_passes(g, K, w.vals[0], reinterpret_cast<int32_t *>(w.keys[0]), g.members);
-    if (e != cudaSuccess) return e;
-    return cudaGetLastError();
-}
-
 // After a stable sort on the upper 32 key bits only: elements whose upper halves agree stand next to each other in
 // their old order; the thread at the head of such a run (they are rare and short: keys are 64-bit hashes) puts it
 // into full-key order by insertion. Runs are disjoint, so the threads do not meet.
@@ -118,6 +95,34 @@ __global__ void k_order_runs(int64_t n, uint64_t *__restrict__ keys, int32_t *__
             vals[b] = va;
         }
     }
+}
+
+cudaError_t launch_partition(Glm &g, int32_t K, uint64_t seed)
+{
+    const int64_t n = g.n_coord;
+    SortWorkspace &w = g.sortws;
+    const int T = 256;
+    k_partition_keys<<<blocks_for(n, T), T, 0, g.stream>>>(n, mix64(seed), w.keys[0], w.vals[0]);
+    int cur = 0;
+    for (int pass = 4; pass < 8; ++pass) { // the upper key halves; equal runs are ordered below
+        cudaError_t e = radix_pass(w.keys[cur], w.vals[cur], w.keys[cur ^ 1], w.vals[cur ^ 1], nullptr, n, 8 * pass,
+                                   w.hist, w.scan_sums, g.stream);
+        if (e != cudaSuccess) return e;
+        cur ^= 1;
+    }
+    {
+        unsigned grid = blocks_for(n, T);
+        if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
+        k_order_runs<<<grid, T, 0, g.stream>>>(n, w.keys[cur], w.vals[cur]);
+    }
+    // an even number of passes: the sorted ids are back in buffer 0
+    k_owner_from_rank<<<blocks_for(n, T), T, 0, g.stream>>>(n, n / K, n % K, w.vals[cur], g.owner);
+    // members: ids 0..n-1 (ascending) stably grouped by owner
+    k_iota<<<blocks_for(n, T), T, 0, g.stream>>>(n, w.vals[0]);
+    // in = vals[0]; scratch = reinterpret keys[0] storage as int32 (keys are dead now)
+    cudaError_t e = owner_passes(g, K, w.vals[0], reinterpret_cast<int32_t *>(w.keys[0]), g.members);
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
 }
 
 cudaError_t launch_permutation(Glm &g, int64_t round, int64_t epochs)
