@@ -44,6 +44,8 @@ def _load():
         lib.orc_mix64.argtypes = [c.c_uint64]
         lib.orc_partition.restype = c.c_int
         lib.orc_partition.argtypes = [c.c_int64, c.c_int32, c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p]
+        lib.orc_partition_sizes.restype = c.c_int
+        lib.orc_partition_sizes.argtypes = [c.c_int64, c.c_int32, c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
         lib.orc_permutation.restype = c.c_int
         lib.orc_permutation.argtypes = [c.c_void_p, c.c_int64, c.c_uint64, c.c_int64, c.c_int64, c.c_void_p]
         lib.orc_step_hinge.restype = c.c_double
@@ -72,14 +74,21 @@ def mix64(x: int) -> int:
     return int(_load().orc_mix64(ctypes.c_uint64(x & (2**64 - 1))))
 
 
-def partition(n: int, K: int, seed: int):
-    """Returns (owner[n] int32, part_off[K+1] int64, members[n] int32)."""
+def partition(n: int, K: int, seed: int, sizes=None):
+    """Returns (owner[n] int32, part_off[K+1] int64, members[n] int32). ``sizes`` (K positive integers summing to n)
+    cuts the same random order into blocks of those sizes instead of equal ones."""
     owner = np.empty(n, np.int32)
     off = np.empty(K + 1, np.int64)
     members = np.empty(n, np.int32)
-    rc = _load().orc_partition(n, K, ctypes.c_uint64(seed & (2**64 - 1)), _p(owner), _p(off), _p(members))
+    if sizes is None:
+        rc = _load().orc_partition(n, K, ctypes.c_uint64(seed & (2**64 - 1)), _p(owner), _p(off), _p(members))
+    else:
+        sz = np.ascontiguousarray(sizes, np.int64)
+        if sz.size != K:
+            raise ValueError("sizes must have K entries")
+        rc = _load().orc_partition_sizes(n, K, ctypes.c_uint64(seed & (2**64 - 1)), _p(sz), _p(owner), _p(off), _p(members))
     if rc != 0:
-        raise ValueError("orc_partition: bad arguments (need 1 <= K <= n)")
+        raise ValueError("orc_partition: bad arguments (need 1 <= K <= n, sizes >= 1 summing to n)")
     return owner, off, members
 
 
@@ -145,8 +154,8 @@ class CocoaOracle:
         self.last_newton_resid = 0.0
 
     # -- a1
-    def partition(self, K: int, seed: int):
-        self.owner, self.part_off, self.members = partition(self.n_coord, K, seed)
+    def partition(self, K: int, seed: int, sizes=None):
+        self.owner, self.part_off, self.members = partition(self.n_coord, K, seed, sizes)
         self.K, self.seed = int(K), int(seed)
 
     def permutation(self, rnd: int, k: int, epoch: int = 0) -> np.ndarray:

@@ -76,16 +76,45 @@ static int orc_i32_cmp(const void *pa, const void *pb)
  * partitions D_k; Sec. 5/6: random assignment of data to tasks). Sort ids by (mix64(mix64(seed) ^ id), id),
  * cut the sorted list into K consecutive blocks, the first n mod K blocks one longer; inside a partition
  * the members are listed in ascending id.  Returns 0, or -1 on bad arguments / out of memory. */
+static int orc_partition_cut(int64_t n, int32_t K, uint64_t seed, const int64_t *sizes, int32_t *owner, int64_t *part_off,
+                             int32_t *members);
+
 int orc_partition(int64_t n, int32_t K, uint64_t seed, int32_t *owner, int64_t *part_off, int32_t *members)
 {
+    return orc_partition_cut(n, K, seed, NULL, owner, part_off, members);
+}
+
+/* The same random order of the coordinates cut into K consecutive blocks of the given sizes (each >= 1, summing to
+ * n): tasks may hold different numbers of samples (Sec. 3, load balancing: data is moved from slow to fast tasks;
+ * Sec. 4.5, rebalancing policy). Returns 0, or -1 on bad arguments / out of memory. */
+int orc_partition_sizes(int64_t n, int32_t K, uint64_t seed, const int64_t *sizes, int32_t *owner, int64_t *part_off,
+                        int32_t *members)
+{
+    if (!sizes) return -1;
+    return orc_partition_cut(n, K, seed, sizes, owner, part_off, members);
+}
+
+static int orc_partition_cut(int64_t n, int32_t K, uint64_t seed, const int64_t *sizes, int32_t *owner, int64_t *part_off,
+                             int32_t *members)
+{
     if (n <= 0 || K <= 0 || (int64_t)K > n) return -1;
+    if (sizes) {
+        int64_t tot = 0;
+        for (int32_t k = 0; k < K; ++k) {
+            if (sizes[k] < 1) return -1;
+            tot += sizes[k];
+        }
+        if (tot != n) return -1;
+    }
     orc_pair *p = (orc_pair *)malloc((size_t)n * sizeof(orc_pair));
     if (!p) return -1;
     const uint64_t s = orc_mix64(seed);
     for (int64_t i = 0; i < n; ++i) { p[i].key = orc_mix64(s ^ (uint64_t)i); p[i].id = (int32_t)i; }
     qsort(p, (size_t)n, sizeof(orc_pair), orc_pair_cmp);
     const int64_t base = n / K, extra = n % K;
-    for (int32_t k = 0; k <= K; ++k) part_off[k] = (int64_t)k * base + (k < extra ? k : extra);
+    part_off[0] = 0;
+    for (int32_t k = 1; k <= K; ++k)
+        part_off[k] = sizes ? part_off[k - 1] + sizes[k - 1] : (int64_t)k * base + (k < extra ? k : extra);
     for (int32_t k = 0; k < K; ++k) {
         for (int64_t pos = part_off[k]; pos < part_off[k + 1]; ++pos) {
             owner[p[pos].id] = k;

@@ -58,6 +58,34 @@ def test_partition_defining_properties(n, K, seed):
         assert hi < lo
 
 
+@pytest.mark.parametrize("n,sizes,seed", [(10, [1, 6, 3], 0), (1000, [400, 1, 99, 500], 3), (64, [64], 5), (7, [1] * 7, 2)])
+def test_partition_with_given_sizes(n, sizes, seed):
+    K = len(sizes)
+    owner, off, members = oracle.partition(n, K, seed, sizes)
+    assert off.tolist() == [0] + np.cumsum(sizes).tolist()                  # the sizes asked for, in order
+    assert sorted(members.tolist()) == list(range(n))                      # disjoint and covering
+    s = py_mix64(seed)
+    keys = [py_mix64(s ^ i) for i in range(n)]
+    order = sorted(range(n), key=lambda i: keys[i])                        # the same random order as the equal split
+    for k in range(K):
+        mk = members[off[k]:off[k + 1]]
+        assert (np.diff(mk) > 0).all() and (owner[mk] == k).all()
+        assert sorted(order[off[k]:off[k + 1]]) == mk.tolist()              # consecutive blocks of that order
+    # equal sizes give the equal split
+    if n % K == 0:
+        o2, off2, m2 = oracle.partition(n, K, seed, [n // K] * K)
+        o1, off1, m1 = oracle.partition(n, K, seed)
+        assert np.array_equal(o1, o2) and np.array_equal(off1, off2) and np.array_equal(m1, m2)
+
+
+def test_partition_rejects_bad_sizes():
+    for sizes in ([5, 6], [0, 10], [11, -1], [3, 3, 3]):
+        with pytest.raises(ValueError):
+            oracle.partition(10, len(sizes), 0, sizes)
+    with pytest.raises(ValueError):
+        oracle.partition(10, 3, 0, [5, 5])
+
+
 def test_partition_rejects_bad_K():
     with pytest.raises(ValueError):
         oracle.partition(5, 6, 0)
@@ -440,6 +468,30 @@ def test_gap_terms_consistency_ascent_and_repartition(loss):
         assert g["primal"] >= g["dual"]
     assert gaps[-1] < 0.25 * gaps[0]
     assert abs(abs(o.state[5]) - (1.0 if loss == "hinge" else 0.5)) < 1e-12      # zero row: a' = 1 / sigmoid(0)
+
+
+def test_unequal_partitions_keep_the_invariants():
+    # tasks of very different sizes (one of a single coordinate): dual ascent for sigma' >= K, a non-negative gap
+    # that shrinks, and v = X^T alpha after every round; repartitioning to equal sizes leaves the state alone
+    n, d, lam, K = 300, 20, 1.0 / 300, 4
+    X, y = dense_problem(n, d, 8)
+    o = CocoaOracle("hinge", "dense", n, d, X, y, lam, threads=2)
+    o.partition(K, 1, sizes=[200, 1, 59, 40])
+    assert np.diff(o.part_off).tolist() == [200, 1, 59, 40]
+    prev_dual, gaps = o.duality_gap()["dual"], []
+    for r in range(20):
+        if r == 10:
+            before = (o.state.copy(), o.v.copy())
+            o.partition(K, 2)
+            assert (o.state == before[0]).all() and (o.v == before[1]).all()
+        o.cocoa_round(0, float(K))
+        g = o.duality_gap(terms=True)
+        assert g["terms"].min() >= -1e-12 and g["dual"] >= prev_dual - 1e-13
+        prev_dual = g["dual"]
+        v2 = o.recompute_shared_vector()
+        assert np.abs(v2 - o.v).max() <= 1e-12 * max(1.0, np.abs(v2).max())
+        gaps.append(g["gap"])
+    assert gaps[-1] < 0.25 * gaps[0]
 
 
 def test_result_is_independent_of_thread_count():
