@@ -107,6 +107,15 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
  * between rounds; keeps alpha, v and the round counter; (re)allocates the per-partition workspaces. */
 chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed);
 
+/* The same, with partitions of given sizes (Sec. 3, load balancing: tasks may hold different numbers of samples, data
+ * moves from slow to fast tasks between iterations; Sec. 4.5, rebalancing policy). The random order of the ids is the
+ * one chicle_partition uses; it is cut into K consecutive blocks of host_sizes[0], ..., host_sizes[K-1] coordinates
+ * (a host array, read during the call; every size >= 1, the sum equal to the number of coordinates, else
+ * CHICLE_ERR_INVALID_ARG and the handle is unchanged). With equal sizes the result is chicle_partition's. A round with
+ * H = 0 then takes as many steps in partition k as it has coordinates; the updates are added as before (every
+ * coordinate has one owner, so no weighting by |D_k| / |D| is needed). */
+chicle_status_t chicle_partition_sizes(chicle_glm_t *h, int32_t K, uint64_t seed, const int64_t *host_sizes);
+
 /* One CoCoA round (Sec. 2.1 Eq. 1, Eq. 2 and worker structure with L = 1; Sec. 5.1: SCD local solver, sigma =
  * number of tasks). Each partition draws this round's seeded visiting order (members ordered by
  * mix64(mix64(seed ^ 0xD1B54A32D192ED03) ^ mix64(round * 2^32 + epoch) ^ id)), walks it strictly in order for H

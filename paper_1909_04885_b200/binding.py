@@ -23,7 +23,7 @@ MEM_HOST, MEM_DEVICE = 0, 1
 
 EXPORTED = ["chicle_glm_create", "chicle_partition", "chicle_cocoa_round", "chicle_duality_gap", "chicle_get_alpha",
             "chicle_get_v", "chicle_get_partition", "chicle_get_permutation", "chicle_set_state", "chicle_get_info",
-            "chicle_last_error", "chicle_glm_destroy", "chicle_partition_noalloc"]
+            "chicle_last_error", "chicle_glm_destroy", "chicle_partition_noalloc", "chicle_partition_sizes"]
 
 
 class ChicleError(RuntimeError):
@@ -67,6 +67,8 @@ def load():
     lib.chicle_glm_create.argtypes = [C.POINTER(Matrix), vp, f32, C.c_int, C.c_int, vp, C.POINTER(Allocator), C.POINTER(vp)]
     lib.chicle_partition.restype = C.c_int
     lib.chicle_partition.argtypes = [vp, i32, u64]
+    lib.chicle_partition_sizes.restype = C.c_int
+    lib.chicle_partition_sizes.argtypes = [vp, i32, u64, vp]
     lib.chicle_cocoa_round.restype = C.c_int
     lib.chicle_cocoa_round.argtypes = [vp, i64, f32, C.POINTER(RoundStats)]
     lib.chicle_duality_gap.restype = C.c_int
@@ -203,8 +205,16 @@ class Glm:
         self.close()
 
     # -- the ABI, one method per entry point
-    def partition(self, K: int, seed: int):
-        self._check(self._lib.chicle_partition(self._h, K, C.c_uint64(seed & (2**64 - 1))))
+    def partition(self, K: int, seed: int, sizes=None):
+        """``chicle_partition``, or ``chicle_partition_sizes`` when ``sizes`` (K positive integers summing to the number
+        of coordinates) is given."""
+        if sizes is None:
+            self._check(self._lib.chicle_partition(self._h, K, C.c_uint64(seed & (2**64 - 1))))
+        else:
+            sz = np.ascontiguousarray(sizes, np.int64)
+            if sz.size != K:
+                raise ValueError("sizes must have K entries")
+            self._check(self._lib.chicle_partition_sizes(self._h, K, C.c_uint64(seed & (2**64 - 1)), _ptr(sz)))
         self.K = K
 
     def cocoa_round(self, H: int = 0, sigma_prime: Optional[float] = None, stats: bool = False):

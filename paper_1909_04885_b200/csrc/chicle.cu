@@ -271,10 +271,18 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
     return CHICLE_OK;
 }
 
-chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed)
+static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed, const int64_t *sizes)
 {
     if (!h) return CHICLE_ERR_INVALID_ARG;
     if (K < 1 || (int64_t)K > h->n_coord) return fail(h, CHICLE_ERR_INVALID_ARG, "need 1 <= K <= number of coordinates");
+    if (sizes) {
+        int64_t tot = 0;
+        for (int32_t k = 0; k < K; ++k) {
+            if (sizes[k] < 1 || sizes[k] > h->n_coord) return fail(h, CHICLE_ERR_INVALID_ARG, "every partition size must be at least 1");
+            tot += sizes[k];
+        }
+        if (tot != h->n_coord) return fail(h, CHICLE_ERR_INVALID_ARG, "the partition sizes must add up to the number of coordinates");
+    }
     cudaError_t e = cudaSetDevice(h->device);
     if (e != cudaSuccess) return fail_cuda(h, e, "cudaSetDevice");
     const int64_t n = h->n_coord;
@@ -324,21 +332,22 @@ chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed)
         delete[] h->h_part_off;
         U = newU; part_off = new_off; h_off = new_hoff;
         // the look-ahead solver's per-round records (their number depends on K); without them the blocked solver runs
-        dev_free(h, h->la_rec); dev_free(h, h->la_dir); dev_free(h, h->la_cursor);
-        h->la_rec = nullptr; h->la_dir = nullptr; h->la_cursor = nullptr; h->la_rec_bytes = 0;
+        dev_free(h, h->la_rec); dev_free(h, h->la_dir); dev_free(h, h->la_cursor); dev_free(h, h->la_blk_base);
+        h->la_rec = nullptr; h->la_dir = nullptr; h->la_cursor = nullptr; h->la_blk_base = nullptr; h->la_rec_bytes = 0;
         const bool dense_fmt = h->fmt == CHICLE_FMT_DENSE_ROWMAJOR;
         if (!dense_fmt || h->dim <= lookahead_max_dense_dim()) {
             size_t rec_bytes = 0, dir_bytes = 0;
             lookahead_workspace(n, h->nnz, K, dense_fmt, h->dim, &rec_bytes, &dir_bytes);
             unsigned char *rec = nullptr, *dir = nullptr;
-            if (alloc_into(h, rec, rec_bytes) && alloc_into(h, dir, dir_bytes) && alloc_into(h, h->la_cursor, 32)) {
+            if (alloc_into(h, rec, rec_bytes) && alloc_into(h, dir, dir_bytes) && alloc_into(h, h->la_cursor, 32) &&
+                alloc_into(h, h->la_blk_base, (size_t)K + 1)) {
                 h->la_rec = rec;
                 h->la_dir = dir;
                 h->la_rec_bytes = rec_bytes;
                 (void)cudaMemsetAsync(h->la_cursor, 0, 32 * sizeof(unsigned long long), h->stream);
             } else {
-                dev_free(h, rec); dev_free(h, dir); dev_free(h, h->la_cursor);
-                h->la_cursor = nullptr;
+                dev_free(h, rec); dev_free(h, dir); dev_free(h, h->la_cursor); dev_free(h, h->la_blk_base);
+                h->la_cursor = nullptr; h->la_blk_base = nullptr;
             }
         }
     }
@@ -346,7 +355,10 @@ chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed)
     h->U = U; h->part_off = part_off; h->h_part_off = h_off;
     h->U_rows = K;
     const int64_t base = n / K, extra = n % K;
-    for (int32_t k = 0; k <= K; ++k) h_off[k] = (int64_t)k * base + (k < extra ? k : extra);
+    h_off[0] = 0;
+    for (int32_t k = 1; k <= K; ++k) h_off[k] = sizes ? h_off[k - 1] + sizes[k - 1] : (int64_t)k * base + (k < extra ? k : extra);
+    h->min_nk = n;
+    for (int32_t k = 0; k < K; ++k) h->min_nk = h_off[k + 1] - h_off[k] < h->min_nk ? h_off[k + 1] - h_off[k] : h->min_nk;
     h->K = K;
     h->seed = seed;
     e = cudaMemcpyAsync(part_off, h_off, ((size_t)K + 1) * 8, cudaMemcpyHostToDevice, h->stream);
@@ -358,6 +370,14 @@ chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed)
     return CHICLE_OK;
 }
 
+chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed) { return partition_impl(h, K, seed, nullptr); }
+
+chicle_status_t chicle_partition_sizes(chicle_glm_t *h, int32_t K, uint64_t seed, const int64_t *host_sizes)
+{
+    if (h && !host_sizes) return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_partition_sizes: sizes is NULL");
+    return partition_impl(h, K, seed, host_sizes);
+}
+
 chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime, chicle_round_stats_t *stats)
 {
     if (!h) return CHICLE_ERR_INVALID_ARG;
@@ -366,7 +386,7 @@ chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime
     if (!(sigma_prime > 0.0f) || !(sigma_prime < 3.0e38f)) return fail(h, CHICLE_ERR_INVALID_ARG, "sigma_prime must be positive and finite");
     cudaError_t e = cudaSetDevice(h->device);
     if (e != cudaSuccess) return fail_cuda(h, e, "cudaSetDevice");
-    const int64_t n = h->n_coord, min_nk = n / h->K;
+    const int64_t n = h->n_coord, min_nk = h->min_nk;
     const int64_t epochs = H == 0 ? 1 : (H + min_nk - 1) / min_nk;
     if (epochs > h->perm_epochs) {
         if (epochs > 1024 || (double)epochs * (double)n * 4.0 > 64e9)

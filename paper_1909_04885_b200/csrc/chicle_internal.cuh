@@ -90,6 +90,7 @@ struct Glm {
     int32_t *members = nullptr; // n_coord, grouped by partition, ascending id inside
     int64_t *part_off = nullptr; // K+1 (device)
     int64_t *h_part_off = nullptr; // K+1 (host)
+    int64_t min_nk = 0;            // smallest partition
     int32_t *perm = nullptr;    // epochs * n_coord
     int64_t perm_epochs = 0;
     float *U = nullptr;         // K * dim: per-partition accumulated update, zero between rounds
@@ -101,6 +102,7 @@ struct Glm {
     void *la_dir = nullptr;
     unsigned long long *la_cursor = nullptr;
     size_t la_rec_bytes = 0;
+    int64_t *la_blk_base = nullptr; // K+1: first block of each partition in this round's numbering of the blocks
     bool time_prepare = false; // record ev[4] between the prepare and the chain kernel (round statistics asked for)
 
     SortWorkspace sortws;

@@ -96,8 +96,8 @@ struct LookParams {
     BlkDir *dir;                // one per block
     unsigned long long *cursor; // [0]: bytes of `rec` handed out so far this round
     unsigned long long rec_cap; // bytes of `rec`
-    int64_t base, extra;        // partition sizes: base + 1 for the first `extra` partitions, base for the rest
-    int64_t nb_long, nb_short;  // blocks of a long / short partition
+    const int64_t *blk_base;    // K + 1: the first block of each partition in this round's numbering of the blocks
+    int32_t K;
     int64_t n_blocks;
 };
 
@@ -108,22 +108,31 @@ struct LookParams {
 #endif
 
 __device__ __forceinline__ int64_t steps_of(const LookParams &P, int64_t nk) { return P.S.H == 0 ? nk : P.S.H; }
-__device__ __forceinline__ int64_t block_base(const LookParams &P, int64_t k)
-{
-    return k < P.extra ? k * P.nb_long : P.extra * P.nb_long + (k - P.extra) * P.nb_short;
-}
+__device__ __forceinline__ int64_t block_base(const LookParams &P, int64_t k) { return P.blk_base[k]; }
 __device__ __forceinline__ void block_to_part(const LookParams &P, int64_t bid, int &k, int64_t &b)
 {
-    const int64_t first = P.extra * P.nb_long;
-    if (bid < first) {
-        k = (int)(bid / P.nb_long);
-        b = bid - (int64_t)k * P.nb_long;
-    } else {
-        const int64_t r = bid - first;
-        const int64_t kk = r / P.nb_short;
-        k = (int)(P.extra + kk);
-        b = r - kk * P.nb_short;
+    int32_t lo = 0, hi = P.K; // blk_base[lo] <= bid < blk_base[hi] (partitions may differ in size)
+    while (hi - lo > 1) {
+        const int32_t mid = (lo + hi) >> 1;
+        if (P.blk_base[mid] <= bid) lo = mid;
+        else hi = mid;
     }
+    k = lo;
+    b = bid - P.blk_base[lo];
+}
+
+// blk_base[k] = blocks of the partitions before k (one thread: K is small next to the work of a round)
+__global__ void k_block_bases(const int64_t *__restrict__ part_off, int32_t K, int64_t H, int64_t *__restrict__ blk_base)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int64_t run = 0;
+    for (int32_t k = 0; k < K; ++k) {
+        blk_base[k] = run;
+        const int64_t nk = part_off[k + 1] - part_off[k];
+        const int64_t steps = H == 0 ? nk : H;
+        run += (steps + kLB - 1) / kLB;
+    }
+    blk_base[K] = run;
 }
 
 // The constants of coordinate c's scalar step (see coordinate_step).
@@ -1046,12 +1055,14 @@ cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
     P.dir = static_cast<BlkDir *>(g.la_dir);
     P.cursor = g.la_cursor;
     P.rec_cap = g.la_rec_bytes;
-    P.base = g.n_coord / g.K;
-    P.extra = g.n_coord % g.K;
-    const int64_t steps_long = S.H == 0 ? P.base + 1 : S.H, steps_short = S.H == 0 ? P.base : S.H;
-    P.nb_long = (steps_long + kLB - 1) / kLB;
-    P.nb_short = (steps_short + kLB - 1) / kLB;
-    P.n_blocks = P.extra * P.nb_long + ((int64_t)g.K - P.extra) * P.nb_short;
+    P.blk_base = g.la_blk_base;
+    P.K = g.K;
+    P.n_blocks = 0;
+    for (int32_t k = 0; k < g.K; ++k) {
+        const int64_t nk = g.h_part_off[k + 1] - g.h_part_off[k];
+        P.n_blocks += ((S.H == 0 ? nk : S.H) + kLB - 1) / kLB;
+    }
+    k_block_bases<<<1, 32, 0, g.stream>>>(g.part_off, g.K, S.H, g.la_blk_base);
     if (P.n_blocks <= 0 || P.n_blocks > 0x7fffffff) return cudaErrorInvalidConfiguration;
     switch (g.loss) {
     case CHICLE_LOSS_HINGE_DUAL: return launch_loss<CHICLE_LOSS_HINGE_DUAL>(g, P);

@@ -30,6 +30,22 @@ __global__ void k_owner_from_rank(int64_t n, int64_t base, int64_t extra, const 
     }
 }
 
+// the same for blocks of given sizes: part_off[k] <= pos < part_off[k + 1]
+__global__ void k_owner_from_offsets(int64_t n, int32_t K, const int64_t *__restrict__ part_off,
+                                     const int32_t *__restrict__ sorted_ids, int32_t *__restrict__ owner)
+{
+    const int64_t pos = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pos < n) {
+        int32_t lo = 0, hi = K; // part_off[lo] <= pos < part_off[hi]
+        while (hi - lo > 1) {
+            const int32_t mid = (lo + hi) >> 1;
+            if (part_off[mid] <= pos) lo = mid;
+            else hi = mid;
+        }
+        owner[sorted_ids[pos]] = lo;
+    }
+}
+
 __global__ void k_iota(int64_t n, int32_t *__restrict__ ids)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -116,7 +132,8 @@ cudaError_t launch_partition(Glm &g, int32_t K, uint64_t seed)
         k_order_runs<<<grid, T, 0, g.stream>>>(n, w.keys[cur], w.vals[cur]);
     }
     // an even number of passes: the sorted ids are back in buffer 0
-    k_owner_from_rank<<<blocks_for(n, T), T, 0, g.stream>>>(n, n / K, n % K, w.vals[cur], g.owner);
+    // (the offsets are on the device already: equal blocks, or the sizes the caller gave)
+    k_owner_from_offsets<<<blocks_for(n, T), T, 0, g.stream>>>(n, K, g.part_off, w.vals[cur], g.owner);
     // members: ids 0..n-1 (ascending) stably grouped by owner
     k_iota<<<blocks_for(n, T), T, 0, g.stream>>>(n, w.vals[0]);
     // in = vals[0]; scratch = reinterpret keys[0] storage as int32 (keys are dead now)

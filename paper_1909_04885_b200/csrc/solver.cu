@@ -386,7 +386,7 @@ cudaError_t launch_local_solver(Glm &g, int64_t H, float sigma_prime, int *varia
     P.inv_n = 1.0f / (float)g.n_examples;
     P.lambda = g.lambda;
     P.sigma = sigma_prime;
-    const int64_t min_nk = g.n_coord / g.K;
+    const int64_t min_nk = g.min_nk;
     P.multi_epoch = (H != 0 && H > min_nk) ? 1 : 0;
 
     const bool dense = g.fmt == CHICLE_FMT_DENSE_ROWMAJOR;

@@ -39,7 +39,7 @@ def check_partition(orc, glm, perm_rounds=(0,)):
             assert np.array_equal(got, orc.permutation(r, k)), "visiting order differs (round %d, k %d)" % (r, k)
 
 
-def run_parity(w, rounds=None, H=None, check_perm=True, resync=False, **kw):
+def run_parity(w, rounds=None, H=None, check_perm=True, resync=False, sizes=None, **kw):
     """Free-running comparison (both sides evolve on their own) unless ``resync``: then the library's state is
     reset to the oracle's before every round, which isolates one round's error."""
     orc, glm = make_pair(w, **kw)
@@ -53,8 +53,8 @@ def run_parity(w, rounds=None, H=None, check_perm=True, resync=False, **kw):
         for r in range(rounds):
             ph = w.phase_at(r)
             if r == 0 or r == ph.start:
-                orc.partition(ph.K, ph.seed)
-                glm.partition(ph.K, ph.seed)
+                orc.partition(ph.K, ph.seed, sizes)
+                glm.partition(ph.K, ph.seed, sizes)
                 if check_perm:
                     check_partition(orc, glm, perm_rounds=(r,))
             if resync and r > 0:

@@ -191,6 +191,44 @@ def test_device_resident_inputs_and_plain_cuda_allocator_give_the_same_bits():
         assert np.array_equal(r[0], res[0][0]) and np.array_equal(r[1], res[0][1]) and r[2] == res[0][2]
 
 
+# ------------------------------------------------------------------ partitions of unequal sizes
+@pytest.mark.parametrize("sizes", [[1, 5000, 2499, 2500], [9000, 1000], [3, 3, 9990, 4]])
+def test_unequal_partitions(sizes):
+    # tasks that hold different numbers of samples: bit-exact partition map and visiting orders, alpha, v and the gap
+    # within tolerance; a partition of one coordinate, and partitions whose last block of 32 steps is ragged
+    w = datagen.make("hinge_csr", 100)
+    w.phases = [Phase(0, len(sizes), 5, float(len(sizes)))]
+    run_parity(w, rounds=4, sizes=sizes)
+
+
+def test_unequal_partitions_dense_ridge_and_partial_H():
+    run_parity(tiny_dense(500, 28, seed=2, loss="logistic", K=3), sizes=[100, 395, 5])
+    w = datagen.make("ridge_csc", 100)
+    K = 4
+    n = w.n_coord
+    w.phases = [Phase(0, K, 1, float(K))]
+    run_parity(w, rounds=3, sizes=[n // 2, n // 4, n // 8, n - n // 2 - n // 4 - n // 8])
+    # a step budget below the smallest partition (one look-ahead pass) and above it (several local epochs)
+    run_parity(tiny_csr(100, 30, seed=5, K=4), H=10, sizes=[12, 40, 30, 18])
+    run_parity(tiny_csr(100, 30, seed=5, K=4), H=30, sizes=[12, 40, 30, 18])
+
+
+def test_partition_sizes_errors_and_equal_sizes():
+    w = tiny_csr(60, 20, seed=1)
+    glm = binding.from_workload(w)
+    try:
+        for bad in ([30, 31], [0, 60], [61, -1]):
+            with pytest.raises(binding.ChicleError) as e:
+                glm.partition(2, 0, bad)
+            assert e.value.status == 1
+        glm.partition(3, 7, [20, 20, 20])
+        a = glm.get_partition().copy()
+        glm.partition(3, 7)
+        assert np.array_equal(a, glm.get_partition())
+    finally:
+        glm.close()
+
+
 # ------------------------------------------------------------------ solver families
 @pytest.mark.parametrize("variant", ["blocked"])
 def test_older_solvers_still_match(variant, monkeypatch):
