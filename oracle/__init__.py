@@ -56,6 +56,10 @@ def _load():
         lib.orc_round.argtypes = [c.c_int, c.c_int64, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int64,
                                   c.c_void_p, c.c_double, c.c_void_p, c.c_void_p, c.c_int32, c.c_void_p,
                                   c.c_void_p, c.c_uint64, c.c_int64, c.c_int64, c.c_double, c.c_int, c.c_void_p]
+        lib.orc_round_steps.restype = c.c_int
+        lib.orc_round_steps.argtypes = [c.c_int, c.c_int64, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int64,
+                                        c.c_void_p, c.c_double, c.c_void_p, c.c_void_p, c.c_int32, c.c_void_p,
+                                        c.c_void_p, c.c_uint64, c.c_int64, c.c_void_p, c.c_double, c.c_int, c.c_void_p]
         lib.orc_gap.restype = c.c_int
         lib.orc_gap.argtypes = [c.c_int, c.c_int64, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int64,
                                 c.c_void_p, c.c_double, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
@@ -162,11 +166,25 @@ class CocoaOracle:
         return permutation(self.members[self.part_off[k]:self.part_off[k + 1]], self.seed, rnd, epoch)
 
     # -- a3..a5
-    def cocoa_round(self, H: int = 0, sigma_prime: Optional[float] = None):
+    def cocoa_round(self, H: int = 0, sigma_prime: Optional[float] = None, steps=None):
+        """One round; ``steps`` (K non-negative integers) gives every partition a step budget of its own instead of H."""
         if self.K == 0:
             raise RuntimeError("partition() first")
         sp = float(self.K if sigma_prime is None else sigma_prime)
         resid = ctypes.c_double(0.0)
+        if steps is not None:
+            st = np.ascontiguousarray(steps, np.int64)
+            if st.size != self.K:
+                raise ValueError("steps must have K entries")
+            rc = _load().orc_round_steps(self.loss, self.n_coord, self.dim, _p(self.indptr), _p(self.indices),
+                                         _p(self.values), self.ld, _p(self.labels), self.lam, _p(self.state), _p(self.v),
+                                         self.K, _p(self.part_off), _p(self.members), ctypes.c_uint64(self.seed),
+                                         self.round, _p(st), sp, self.threads, ctypes.byref(resid))
+            if rc != 0:
+                raise RuntimeError("orc_round_steps failed")
+            self.last_newton_resid = resid.value
+            self.round += 1
+            return
         rc = _load().orc_round(self.loss, self.n_coord, self.dim, _p(self.indptr), _p(self.indices),
                                _p(self.values), self.ld, _p(self.labels), self.lam, _p(self.state), _p(self.v),
                                self.K, _p(self.part_off), _p(self.members), ctypes.c_uint64(self.seed),

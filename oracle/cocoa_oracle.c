@@ -316,10 +316,41 @@ static int orc_local_solver(int loss, const orc_mat *A, const float *labels, dou
  * same v, then v += sum_k dv_k with k ascending.  H = 0 means one local epoch (n_k steps).
  * newton_resid (nullable) receives the largest |g| left by a logistic step in this round.
  * Returns 0 on success, -1 on bad arguments or allocation failure. */
+static int orc_round_impl(int loss, int64_t n_coord, int64_t dim, const int64_t *indptr, const int32_t *indices,
+                          const float *values, int64_t ld, const float *labels, double lambda,
+                          double *state, double *v, int32_t K, const int64_t *part_off, const int32_t *members,
+                          uint64_t seed, int64_t round, int64_t H, const int64_t *steps_k, double sigma_p, int nthreads,
+                          double *newton_resid);
+
 int orc_round(int loss, int64_t n_coord, int64_t dim, const int64_t *indptr, const int32_t *indices,
               const float *values, int64_t ld, const float *labels, double lambda,
               double *state, double *v, int32_t K, const int64_t *part_off, const int32_t *members,
               uint64_t seed, int64_t round, int64_t H, double sigma_p, int nthreads, double *newton_resid)
+{
+    return orc_round_impl(loss, n_coord, dim, indptr, indices, values, ld, labels, lambda, state, v, K, part_off, members,
+                          seed, round, H, NULL, sigma_p, nthreads, newton_resid);
+}
+
+/* The same round with a step budget of its own for every partition (Sec. 3, load balancing: a task processes a
+ * number of samples per iteration that suits its speed): partition k takes steps_k[k] >= 0 coordinate steps of its
+ * visiting order (0: it sits the round out). */
+int orc_round_steps(int loss, int64_t n_coord, int64_t dim, const int64_t *indptr, const int32_t *indices,
+                    const float *values, int64_t ld, const float *labels, double lambda,
+                    double *state, double *v, int32_t K, const int64_t *part_off, const int32_t *members,
+                    uint64_t seed, int64_t round, const int64_t *steps_k, double sigma_p, int nthreads, double *newton_resid)
+{
+    if (!steps_k) return -1;
+    for (int32_t k = 0; k < K; ++k)
+        if (steps_k[k] < 0) return -1;
+    return orc_round_impl(loss, n_coord, dim, indptr, indices, values, ld, labels, lambda, state, v, K, part_off, members,
+                          seed, round, 0, steps_k, sigma_p, nthreads, newton_resid);
+}
+
+static int orc_round_impl(int loss, int64_t n_coord, int64_t dim, const int64_t *indptr, const int32_t *indices,
+                          const float *values, int64_t ld, const float *labels, double lambda,
+                          double *state, double *v, int32_t K, const int64_t *part_off, const int32_t *members,
+                          uint64_t seed, int64_t round, int64_t H, const int64_t *steps_k, double sigma_p, int nthreads,
+                          double *newton_resid)
 {
     if (K <= 0 || n_coord <= 0 || dim <= 0 || lambda <= 0.0 || sigma_p <= 0.0 || H < 0) return -1;
     orc_mat A = { n_coord, dim, ld, indptr, indices, values };
@@ -338,7 +369,8 @@ int orc_round(int loss, int64_t n_coord, int64_t dim, const int64_t *indptr, con
         double *vloc = (double *)malloc((size_t)dim * sizeof(double));
         if (!vloc) { rc_k[k] = -1; continue; }
         memcpy(vloc, v, (size_t)dim * sizeof(double));
-        const int64_t steps = (H == 0) ? n_k : H;
+        const int64_t steps = steps_k ? steps_k[k] : ((H == 0) ? n_k : H);
+        if (steps == 0) continue;
         rc_k[k] = orc_local_solver(loss, &A, labels, lambda, scale_n, state, members + part_off[k], n_k, seed,
                                    round, steps, sigma_p, vloc, dv_all + (size_t)k * (size_t)dim, &resid_k[k]);
         free(vloc);

@@ -494,6 +494,37 @@ def test_unequal_partitions_keep_the_invariants():
     assert gaps[-1] < 0.5 * gaps[0]
 
 
+def test_step_budgets_per_partition():
+    # budgets equal to H reproduce the round with H; a budget of 0 leaves the partition's coordinates alone; the
+    # invariants hold with ragged budgets
+    n, d, K = 240, 12, 3
+    X, y = dense_problem(n, d, 13)
+    a = CocoaOracle("hinge", "dense", n, d, X, y, 1.0 / n, threads=2)
+    b = CocoaOracle("hinge", "dense", n, d, X, y, 1.0 / n, threads=2)
+    a.partition(K, 4)
+    b.partition(K, 4)
+    a.cocoa_round(50, 3.0)
+    b.cocoa_round(0, 3.0, steps=[50, 50, 50])
+    assert (a.state == b.state).all() and (a.v == b.v).all()
+    a.cocoa_round(0, 3.0)
+    b.cocoa_round(0, 3.0, steps=np.diff(b.part_off))
+    assert (a.state == b.state).all() and (a.v == b.v).all()
+    before = b.state.copy()
+    prev = b.duality_gap()["dual"]
+    b.cocoa_round(0, 3.0, steps=[80, 0, 7])
+    idle = b.members[b.part_off[1]:b.part_off[2]]
+    assert (b.state[idle] == before[idle]).all()
+    busy0 = b.members[b.part_off[0]:b.part_off[1]]
+    assert (b.state[busy0] != before[busy0]).any()
+    assert np.count_nonzero(b.state[b.members[b.part_off[2]:]] != before[b.members[b.part_off[2]:]]) <= 7
+    g = b.duality_gap(terms=True)
+    assert g["dual"] >= prev - 1e-13 and g["terms"].min() >= -1e-12
+    v2 = b.recompute_shared_vector()
+    assert np.abs(v2 - b.v).max() <= 1e-12 * max(1.0, np.abs(v2).max())
+    with pytest.raises(RuntimeError):
+        b.cocoa_round(0, 3.0, steps=[1, -1, 1])
+
+
 def test_result_is_independent_of_thread_count():
     n, d = 300, 10
     X, y = dense_problem(n, d, 4)
