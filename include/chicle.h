@@ -125,6 +125,16 @@ chicle_status_t chicle_partition_sizes(chicle_glm_t *h, int32_t K, uint64_t seed
  * which case the stream is synchronised and *stats filled. */
 chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime, chicle_round_stats_t *stats);
 
+/* The same round with a step budget per partition (Sec. 3: the number of samples a task processes in an iteration is
+ * set per task, so that slow and fast tasks finish together; Sec. 4.5). Partition k takes host_steps[k] coordinate
+ * steps along the first host_steps[k] entries of the visiting order that chicle_cocoa_round would walk this round
+ * (a host array of K entries, read during the call; 0 <= host_steps[k] <= size of partition k, else
+ * CHICLE_ERR_INVALID_ARG and nothing is enqueued). A partition with budget 0 sits the round out; with every budget
+ * equal to H (or to the partition's size) the result is chicle_cocoa_round's with that H (or H = 0), bit for bit.
+ * The round counter advances even if every budget is 0. stats->steps is the sum of the budgets. */
+chicle_status_t chicle_cocoa_round_steps(chicle_glm_t *h, const int64_t *host_steps, float sigma_prime,
+                                         chicle_round_stats_t *stats);
+
 /* Duality gap P(w(alpha)) - D(alpha) of the current state (Sec. 4.1, Sec. 5: the metric solvers report), with
  * fp64 accumulation in a fixed order. host_gap / host_primal / host_dual may each be NULL. Synchronises. */
 chicle_status_t chicle_duality_gap(chicle_glm_t *h, double *host_gap, double *host_primal, double *host_dual);

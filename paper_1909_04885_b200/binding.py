@@ -23,7 +23,8 @@ MEM_HOST, MEM_DEVICE = 0, 1
 
 EXPORTED = ["chicle_glm_create", "chicle_partition", "chicle_cocoa_round", "chicle_duality_gap", "chicle_get_alpha",
             "chicle_get_v", "chicle_get_partition", "chicle_get_permutation", "chicle_set_state", "chicle_get_info",
-            "chicle_last_error", "chicle_glm_destroy", "chicle_partition_noalloc", "chicle_partition_sizes"]
+            "chicle_last_error", "chicle_glm_destroy", "chicle_partition_noalloc", "chicle_partition_sizes",
+            "chicle_cocoa_round_steps"]
 
 
 class ChicleError(RuntimeError):
@@ -71,6 +72,8 @@ def load():
     lib.chicle_partition_sizes.argtypes = [vp, i32, u64, vp]
     lib.chicle_cocoa_round.restype = C.c_int
     lib.chicle_cocoa_round.argtypes = [vp, i64, f32, C.POINTER(RoundStats)]
+    lib.chicle_cocoa_round_steps.restype = C.c_int
+    lib.chicle_cocoa_round_steps.argtypes = [vp, vp, f32, C.POINTER(RoundStats)]
     lib.chicle_duality_gap.restype = C.c_int
     lib.chicle_duality_gap.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     for name in ("chicle_get_alpha", "chicle_get_v"):
@@ -217,15 +220,22 @@ class Glm:
             self._check(self._lib.chicle_partition_sizes(self._h, K, C.c_uint64(seed & (2**64 - 1)), _ptr(sz)))
         self.K = K
 
-    def cocoa_round(self, H: int = 0, sigma_prime: Optional[float] = None, stats: bool = False):
+    def cocoa_round(self, H: int = 0, sigma_prime: Optional[float] = None, stats: bool = False, steps=None):
+        """One round; ``steps`` (K integers, 0 <= steps[k] <= size of partition k) gives each partition its own budget."""
         sp = float(self.K if sigma_prime is None else sigma_prime)
+        rs = RoundStats() if stats else None
+        ref = C.byref(rs) if stats else None
+        if steps is not None:
+            st = np.ascontiguousarray(steps, np.int64)
+            if st.size != self.K:
+                raise ValueError("steps must have K entries")
+            self._check(self._lib.chicle_cocoa_round_steps(self._h, st.ctypes.data, C.c_float(sp), ref))
+        else:
+            self._check(self._lib.chicle_cocoa_round(self._h, H, C.c_float(sp), ref))
         if stats:
-            rs = RoundStats()
-            self._check(self._lib.chicle_cocoa_round(self._h, H, C.c_float(sp), C.byref(rs)))
             return {"ms_permutation": rs.ms_permutation, "ms_local": rs.ms_local, "ms_reduce": rs.ms_reduce,
                     "ms_total": rs.ms_total, "steps": rs.steps, "solver_variant": rs.solver_variant,
                     "ms_prepare": rs.ms_prepare}
-        self._check(self._lib.chicle_cocoa_round(self._h, H, C.c_float(sp), None))
         return None
 
     def duality_gap(self):

@@ -320,7 +320,7 @@ static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed,
         // release the old update workspace first: at the large configurations two of them do not fit
         dev_free(h, h->U);
         h->U = nullptr;
-        bool ok = new_hoff && alloc_into(h, newU, (size_t)K * (size_t)h->dim) && alloc_into(h, new_off, (size_t)K + 1);
+        bool ok = new_hoff && alloc_into(h, newU, (size_t)K * (size_t)h->dim) && alloc_into(h, new_off, 2 * (size_t)K + 2); // K+1 offsets, then K step budgets
         if (!ok) {
             delete[] new_hoff;
             dev_free(h, newU); dev_free(h, new_off);
@@ -353,6 +353,7 @@ static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed,
     }
     if (fresh) { h->owner = owner; h->members = members; h->perm = perm; h->perm_epochs = 1; }
     h->U = U; h->part_off = part_off; h->h_part_off = h_off;
+    h->d_steps = part_off + K + 1;
     h->U_rows = K;
     const int64_t base = n / K, extra = n % K;
     h_off[0] = 0;
@@ -378,12 +379,21 @@ chicle_status_t chicle_partition_sizes(chicle_glm_t *h, int32_t K, uint64_t seed
     return partition_impl(h, K, seed, host_sizes);
 }
 
-chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime, chicle_round_stats_t *stats)
+// One round. host_steps == nullptr: every partition takes H steps (0: one local epoch). Otherwise partition k takes
+// host_steps[k] steps (H is 0 then).
+static chicle_status_t round_impl(chicle_glm_t *h, int64_t H, const int64_t *host_steps, float sigma_prime, chicle_round_stats_t *stats)
 {
-    if (!h) return CHICLE_ERR_INVALID_ARG;
     if (h->K <= 0) return fail(h, CHICLE_ERR_BAD_STATE, "chicle_partition must be called before chicle_cocoa_round");
     if (H < 0) return fail(h, CHICLE_ERR_INVALID_ARG, "H must be >= 0");
     if (!(sigma_prime > 0.0f) || !(sigma_prime < 3.0e38f)) return fail(h, CHICLE_ERR_INVALID_ARG, "sigma_prime must be positive and finite");
+    int64_t budget_total = 0;
+    if (host_steps) {
+        for (int32_t k = 0; k < h->K; ++k) {
+            if (host_steps[k] < 0 || host_steps[k] > h->h_part_off[k + 1] - h->h_part_off[k])
+                return fail(h, CHICLE_ERR_INVALID_ARG, "a partition's step budget must lie between 0 and its size");
+            budget_total += host_steps[k];
+        }
+    }
     cudaError_t e = cudaSetDevice(h->device);
     if (e != cudaSuccess) return fail_cuda(h, e, "cudaSetDevice");
     const int64_t n = h->n_coord, min_nk = h->min_nk;
@@ -406,7 +416,15 @@ chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime
     if (stats) (void)cudaEventRecord(h->ev[1], s);
     int variant = 0;
     h->time_prepare = stats != nullptr;
-    e = launch_local_solver(*h, H, sigma_prime, &variant);
+    if (host_steps) {
+        // a pageable source: the runtime has taken its copy of the K words when the call returns
+        e = cudaMemcpyAsync(h->d_steps, host_steps, (size_t)h->K * sizeof(int64_t), cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return fail_cuda(h, e, "step budgets to the device");
+        h->round_steps = host_steps;
+    }
+    if (!host_steps || budget_total > 0) e = launch_local_solver(*h, H, sigma_prime, &variant);
+    else if (stats) (void)cudaEventRecord(h->ev[4], s); // nobody steps this round
+    h->round_steps = nullptr;
     if (e != cudaSuccess) return fail_cuda(h, e, "local solver launch");
     if (stats) (void)cudaEventRecord(h->ev[2], s);
     e = launch_reduce(*h);
@@ -425,7 +443,7 @@ chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime
         int64_t steps = 0;
         for (int32_t k = 0; k < h->K; ++k) {
             const int64_t nk = h->h_part_off[k + 1] - h->h_part_off[k];
-            steps += nk <= 0 ? 0 : (H == 0 ? nk : H);
+            steps += host_steps ? host_steps[k] : (nk <= 0 ? 0 : (H == 0 ? nk : H));
         }
         r.steps = steps;
         r.solver_variant = variant;
@@ -433,6 +451,19 @@ chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime
         *stats = r;
     }
     return CHICLE_OK;
+}
+
+chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime, chicle_round_stats_t *stats)
+{
+    if (!h) return CHICLE_ERR_INVALID_ARG;
+    return round_impl(h, H, nullptr, sigma_prime, stats);
+}
+
+chicle_status_t chicle_cocoa_round_steps(chicle_glm_t *h, const int64_t *host_steps, float sigma_prime, chicle_round_stats_t *stats)
+{
+    if (!h) return CHICLE_ERR_INVALID_ARG;
+    if (!host_steps) return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_cocoa_round_steps: steps is NULL");
+    return round_impl(h, 0, host_steps, sigma_prime, stats);
 }
 
 chicle_status_t chicle_duality_gap(chicle_glm_t *h, double *host_gap, double *host_primal, double *host_dual)

@@ -91,6 +91,8 @@ struct Glm {
     int64_t *part_off = nullptr; // K+1 (device)
     int64_t *h_part_off = nullptr; // K+1 (host)
     int64_t min_nk = 0;            // smallest partition
+    int64_t *d_steps = nullptr;    // K (device, behind part_off): the step budgets of a round that gives each partition its own
+    const int64_t *round_steps = nullptr; // the same on the host while such a round is being enqueued, else nullptr
     int32_t *perm = nullptr;    // epochs * n_coord
     int64_t perm_epochs = 0;
     float *U = nullptr;         // K * dim: per-partition accumulated update, zero between rounds

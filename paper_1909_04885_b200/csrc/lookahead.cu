@@ -107,7 +107,7 @@ struct LookParams {
 #define LA_T(acc) do { } while (0)
 #endif
 
-__device__ __forceinline__ int64_t steps_of(const LookParams &P, int64_t nk) { return P.S.H == 0 ? nk : P.S.H; }
+__device__ __forceinline__ int64_t steps_of(const LookParams &P, int64_t k, int64_t nk) { return partition_steps(P.S, k, nk); }
 __device__ __forceinline__ int64_t block_base(const LookParams &P, int64_t k) { return P.blk_base[k]; }
 __device__ __forceinline__ void block_to_part(const LookParams &P, int64_t bid, int &k, int64_t &b)
 {
@@ -122,14 +122,13 @@ __device__ __forceinline__ void block_to_part(const LookParams &P, int64_t bid, 
 }
 
 // blk_base[k] = blocks of the partitions before k (one thread: K is small next to the work of a round)
-__global__ void k_block_bases(const int64_t *__restrict__ part_off, int32_t K, int64_t H, int64_t *__restrict__ blk_base)
+__global__ void k_block_bases(SolverParams S, int32_t K, int64_t *__restrict__ blk_base)
 {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     int64_t run = 0;
     for (int32_t k = 0; k < K; ++k) {
         blk_base[k] = run;
-        const int64_t nk = part_off[k + 1] - part_off[k];
-        const int64_t steps = H == 0 ? nk : H;
+        const int64_t steps = partition_steps(S, k, S.part_off[k + 1] - S.part_off[k]);
         run += (steps + kLB - 1) / kLB;
     }
     blk_base[K] = run;
@@ -257,7 +256,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) k_lookahead_prepare(c
     block_to_part(P, bid, k, b);
     const int64_t off = P.S.part_off[k];
     const int64_t nk = P.S.part_off[k + 1] - off;
-    const int64_t steps = steps_of(P, nk);
+    const int64_t steps = steps_of(P, k, nk);
     const int cnt = (int)((steps - b * kLB) < kLB ? (steps - b * kLB) : kLB);
 #ifdef CHICLE_LA_TIMING
     long long pt0 = clock64(), pt1 = 0;
@@ -500,7 +499,7 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
     block_to_part(P, bid, k, b);
     const int64_t off = P.S.part_off[k];
     const int64_t nk = P.S.part_off[k + 1] - off;
-    const int64_t steps = steps_of(P, nk);
+    const int64_t steps = steps_of(P, k, nk);
     const int cnt = (int)((steps - b * kLB) < kLB ? (steps - b * kLB) : kLB);
     const int dim = (int)P.S.dim;
     if (tid == 0) {
@@ -582,7 +581,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
     const SolverParams &S = P.S;
 
     const int64_t nk = S.part_off[k + 1] - S.part_off[k];
-    const int64_t steps = steps_of(P, nk);
+    const int64_t steps = steps_of(P, k, nk);
     const int64_t nblocks = (steps + kLB - 1) / kLB;
     const int64_t bid0 = block_base(P, k);
     float *Uk = S.U + (size_t)k * (size_t)S.dim;
@@ -1060,9 +1059,10 @@ cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
     P.n_blocks = 0;
     for (int32_t k = 0; k < g.K; ++k) {
         const int64_t nk = g.h_part_off[k + 1] - g.h_part_off[k];
-        P.n_blocks += ((S.H == 0 ? nk : S.H) + kLB - 1) / kLB;
+        const int64_t steps = g.round_steps ? g.round_steps[k] : (S.H == 0 ? nk : S.H);
+        P.n_blocks += (steps + kLB - 1) / kLB;
     }
-    k_block_bases<<<1, 32, 0, g.stream>>>(g.part_off, g.K, S.H, g.la_blk_base);
+    k_block_bases<<<1, 32, 0, g.stream>>>(S, g.K, g.la_blk_base);
     if (P.n_blocks <= 0 || P.n_blocks > 0x7fffffff) return cudaErrorInvalidConfiguration;
     switch (g.loss) {
     case CHICLE_LOSS_HINGE_DUAL: return launch_loss<CHICLE_LOSS_HINGE_DUAL>(g, P);

@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(32 * (1 + kProdWarps), 1) k_local_scd(const So
 
     const int64_t off = P.part_off[k];
     const int64_t nk = P.part_off[k + 1] - off;
-    const int64_t steps = nk <= 0 ? 0 : (P.H == 0 ? nk : P.H);
+    const int64_t steps = partition_steps(P, k, nk);
 
     if (threadIdx.x == 0) {
         *progress = 0;
@@ -382,6 +382,7 @@ cudaError_t launch_local_solver(Glm &g, int64_t H, float sigma_prime, int *varia
     P.n_coord = g.n_coord;
     P.dim = g.dim;
     P.H = H;
+    P.steps_k = g.round_steps ? g.d_steps : nullptr;
     P.lam_n = g.lambda * (float)g.n_examples;
     P.inv_n = 1.0f / (float)g.n_examples;
     P.lambda = g.lambda;

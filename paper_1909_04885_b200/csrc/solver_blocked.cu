@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) k_local_scd_blocked(const Solver
 
     const int64_t off = P.part_off[k];
     const int64_t nk = P.part_off[k + 1] - off;
-    const int64_t steps = nk <= 0 ? 0 : (P.H == 0 ? nk : P.H);
+    const int64_t steps = partition_steps(P, k, nk);
     float *Uk = P.U + (size_t)k * (size_t)P.dim;
     const int hot_n = HOT < P.dim ? HOT : (int)P.dim; // ids below hot_n live in the direct part of W
     const float inv_sigma = 1.0f / P.sigma;

@@ -109,9 +109,18 @@ struct SolverParams {
     const int32_t *perm; // epochs x n_coord
     uint32_t *status;
     int64_t n_coord, dim, H;
+    const int64_t *steps_k; // K step budgets of this round, one per partition (each at most its size), or nullptr: H rules
     float lam_n, inv_n, lambda, sigma;
     int cap, nslot, multi_epoch;
 };
+
+// Coordinate steps partition k (of nk coordinates) takes this round.
+__device__ __forceinline__ int64_t partition_steps(const SolverParams &P, int64_t k, int64_t nk)
+{
+    if (nk <= 0) return 0;
+    if (P.steps_k) return P.steps_k[k];
+    return P.H == 0 ? nk : P.H;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t a, uint32_t count)

@@ -39,8 +39,9 @@ def check_partition(orc, glm, perm_rounds=(0,)):
             assert np.array_equal(got, orc.permutation(r, k)), "visiting order differs (round %d, k %d)" % (r, k)
 
 
-def run_parity(w, rounds=None, H=None, check_perm=True, resync=False, sizes=None, **kw):
-    """Free-running comparison (both sides evolve on their own) unless ``resync``: then the library's state is
+def run_parity(w, rounds=None, H=None, check_perm=True, resync=False, sizes=None, steps=None, **kw):
+    """``steps``: a function of the round that returns the K step budgets of that round (instead of H).
+    Free-running comparison (both sides evolve on their own) unless ``resync``: then the library's state is
     reset to the oracle's before every round, which isolates one round's error."""
     orc, glm = make_pair(w, **kw)
     rounds = w.rounds if rounds is None else rounds
@@ -59,8 +60,12 @@ def run_parity(w, rounds=None, H=None, check_perm=True, resync=False, sizes=None
                     check_partition(orc, glm, perm_rounds=(r,))
             if resync and r > 0:
                 glm.set_state(orc.state.astype(np.float32), orc.v.astype(np.float32), orc.round)
-            orc.cocoa_round(H, ph.sigma_prime)
-            glm.cocoa_round(H, ph.sigma_prime)
+            if steps is not None:
+                orc.cocoa_round(0, ph.sigma_prime, steps=steps(r))
+                glm.cocoa_round(0, ph.sigma_prime, steps=steps(r))
+            else:
+                orc.cocoa_round(H, ph.sigma_prime)
+                glm.cocoa_round(H, ph.sigma_prime)
             ea, ev = rel_l2(glm.get_alpha(), orc.state), rel_l2(glm.get_v(), orc.v)
             worst["alpha"], worst["v"] = max(worst["alpha"], ea), max(worst["v"], ev)
             assert ea <= REL_TOL, "round %d: alpha rel err %.3e" % (r, ea)

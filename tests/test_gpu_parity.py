@@ -213,6 +213,52 @@ def test_unequal_partitions_dense_ridge_and_partial_H():
     run_parity(tiny_csr(100, 30, seed=5, K=4), H=30, sizes=[12, 40, 30, 18])
 
 
+def test_step_budgets_per_partition(monkeypatch):
+    # Sec. 3: every task gets the number of samples per iteration that suits its speed. Budgets that change from round
+    # to round, ragged against the 32-step blocks, with partitions that sit a round out.
+    sizes = [12, 40, 30, 18]
+    table = [[12, 40, 30, 18], [5, 33, 0, 18], [0, 1, 30, 7], [0, 0, 0, 0], [12, 0, 0, 0]]
+    w = tiny_csr(100, 30, seed=5, K=4)
+    run_parity(w, rounds=5, sizes=sizes, steps=lambda r: table[r])
+    w = datagen.make("hinge_csr", 100)
+    K = w.phases[0].K
+    n = w.n_coord
+    base = np.diff(np.linspace(0, n, K + 1).astype(np.int64))
+    budget = lambda r: [int(b) // (1 + (k + r) % 3) if (k + r) % 5 else 0 for k, b in enumerate(base)]
+    run_parity(w, rounds=4, sizes=[int(b) for b in base], steps=budget)
+    run_parity(tiny_dense(500, 28, seed=2, loss="logistic", K=3), sizes=[100, 395, 5], steps=lambda r: [100 - 33 * r, 64 + r, r])
+    w = datagen.make("ridge_csc", 100)
+    w.phases = [Phase(0, 4, 1, 4.0)]
+    n = w.n_coord
+    run_parity(w, rounds=3, steps=lambda r: [n // 4 - r, 31, 32 * r, n // 8])
+    monkeypatch.setenv("CHICLE_FORCE_VARIANT", "blocked")
+    run_parity(tiny_csr(100, 30, seed=5, K=4), rounds=5, sizes=sizes, steps=lambda r: table[r])
+
+
+def test_step_budgets_equal_to_H_reproduce_the_round_and_bad_budgets_are_refused():
+    w = tiny_csr(300, 40, seed=3, K=3)
+    a, b = binding.from_workload(w), binding.from_workload(w)
+    try:
+        a.partition(3, 1)
+        b.partition(3, 1)
+        a.cocoa_round(37, 3.0)
+        st = b.cocoa_round(0, 3.0, stats=True, steps=[37, 37, 37])
+        assert st["steps"] == 111
+        assert np.array_equal(a.get_alpha(), b.get_alpha()) and np.array_equal(a.get_v(), b.get_v())
+        a.cocoa_round(0, 3.0)
+        b.cocoa_round(0, 3.0, steps=[100, 100, 100])
+        assert np.array_equal(a.get_alpha(), b.get_alpha()) and np.array_equal(a.get_v(), b.get_v())
+        before = b.get_alpha().copy()
+        for bad in ([101, 1, 1], [-1, 1, 1]):
+            with pytest.raises(binding.ChicleError) as e:
+                b.cocoa_round(0, 3.0, steps=bad)
+            assert e.value.status == 1
+        assert np.array_equal(before, b.get_alpha()) and b.info()["round"] == 2
+    finally:
+        a.close()
+        b.close()
+
+
 def test_partition_sizes_errors_and_equal_sizes():
     w = tiny_csr(60, 20, seed=1)
     glm = binding.from_workload(w)
