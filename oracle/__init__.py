@@ -162,6 +162,13 @@ class CocoaOracle:
         self.owner, self.part_off, self.members = partition(self.n_coord, K, seed, sizes)
         self.K, self.seed = int(K), int(seed)
 
+    def partition_chunks(self, K: int, seed: int, chunk_off, chunk_task):
+        """The partition that a placement of data chunks on K tasks induces (Sec. 3, Sec. 4.3); ``seed`` keys the
+        visiting orders of the rounds that follow."""
+        from . import chunks
+        self.owner, self.part_off, self.members = chunks.partition_from_chunks(self.n_coord, K, chunk_off, chunk_task)
+        self.K, self.seed = int(K), int(seed)
+
     def permutation(self, rnd: int, k: int, epoch: int = 0) -> np.ndarray:
         return permutation(self.members[self.part_off[k]:self.part_off[k + 1]], self.seed, rnd, epoch)
 
