@@ -116,6 +116,55 @@ chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed);
  * coordinate has one owner, so no weighting by |D_k| / |D| is needed). */
 chicle_status_t chicle_partition_sizes(chicle_glm_t *h, int32_t K, uint64_t seed, const int64_t *host_sizes);
 
+/* ---- mobile data chunks (Sec. 3 core concepts: the samples live in many small fixed-size chunks that the scheduler
+ * moves between immobile tasks; Sec. 4.3: a chunk holds samples and their per-sample state, their number varies with
+ * their size). The five functions below are host-side integer logic: all pointers are HOST arrays, no GPU is touched,
+ * no handle is needed. A placement is `chunk_off` (n_chunks + 1 ascending coordinate offsets, chunk c = coordinates
+ * chunk_off[c] .. chunk_off[c+1]-1 in id order) and `chunk_task` (n_chunks task numbers). The paper fixes none of the
+ * integer rules; the ones stated here are this library's. ---- */
+
+/* Cuts the coordinates into chunks of at most chunk_bytes: coordinate i occupies 8 bytes per stored entry (sparse:
+ * host_indptr[i+1] - host_indptr[i] entries; dense: host_indptr NULL and 4 * dense_dim bytes instead) plus 8 bytes of
+ * state; a chunk is closed in front of the coordinate that would take it above chunk_bytes and holds at least one
+ * coordinate. host_chunk_off needs room for n_coord + 1 entries. Returns the number of chunks, or -1 on bad arguments. */
+int64_t chicle_chunks_cut(int64_t n_coord, const int64_t *host_indptr, int64_t dense_dim, int64_t chunk_bytes,
+                          int64_t *host_chunk_off);
+
+/* First placement (Sec. 6: data is assigned to tasks at random): the chunks, ordered by (mix64(mix64(seed) ^ chunk),
+ * chunk), are dealt in K consecutive runs, the first n_chunks mod K tasks getting one more. 1 <= K <= n_chunks. */
+chicle_status_t chicle_chunks_assign(int64_t n_chunks, int32_t K, uint64_t seed, int32_t *host_chunk_task);
+
+/* Scale-in (Sec. 4.5 elastic scaling policy: the chunks of to-be-freed tasks are redistributed round-robin): tasks
+ * K_new .. K_old-1 are freed; their chunks, in ascending chunk number, go to tasks 0, 1, .., K_new-1, 0, .. in turn.
+ * No other chunk moves. In place. 1 <= K_new <= K_old. */
+chicle_status_t chicle_chunks_scale_in(int64_t n_chunks, int32_t K_old, int32_t K_new, int32_t *host_chunk_task);
+
+/* Scale-out (Sec. 4.5; Sec. 5.3: the chunks moved to new tasks are picked at random from every old task, which
+ * reshuffles the samples): old task j, holding m_j chunks, gives away floor(m_j * (K_new - K_old) / K_new) of them,
+ * the first ones in the order (mix64(mix64(seed ^ 0xA0761D6478BD642F) ^ chunk), chunk); the chunks given away are
+ * dealt to tasks K_old .. K_new-1 in turn, old tasks in ascending order, the turn carrying over. No other chunk
+ * moves. In place. 1 <= K_old <= K_new; a task number outside [0, K_old) on entry: CHICLE_ERR_INVALID_ARG. */
+chicle_status_t chicle_chunks_scale_out(int64_t n_chunks, int32_t K_old, int32_t K_new, uint64_t seed,
+                                        int32_t *host_chunk_task);
+
+/* One step of the rebalancing policy (Sec. 4.5: chunks move gradually from slower to faster tasks until the
+ * difference is below one chunk's processing time). host_time_per_sample[k] is task k's time per sample (the caller's
+ * median over its window). A task's round time is its samples times that. The task with the longest round time (ties:
+ * lowest number) gives its highest-numbered chunk to the task with the shortest (ties: lowest number), unless the two
+ * times differ by no more than that chunk's processing time on the slow task, or the slow task holds one chunk only.
+ * Returns 1 if a chunk moved, 0 if not, -1 on bad arguments. */
+int chicle_chunks_rebalance_step(int64_t n_chunks, const int64_t *host_chunk_off, int32_t K,
+                                 const double *host_time_per_sample, int32_t *host_chunk_task);
+
+/* The partition a placement induces: coordinate i belongs to the task of its chunk; members in ascending id order
+ * inside a partition (the owner map and the member lists are built on the device). Otherwise as chicle_partition:
+ * legal between rounds, keeps alpha, v and the round counter (the state moves with the samples, Sec. 4.3); `seed` keys
+ * the visiting orders of the rounds that follow. K <= n_chunks <= coordinates, offsets from 0 to the number of
+ * coordinates and strictly increasing, tasks in [0, K), every task holding a chunk: else CHICLE_ERR_INVALID_ARG and
+ * the handle is unchanged. The host arrays are read during the call. */
+chicle_status_t chicle_partition_chunks(chicle_glm_t *h, int32_t K, uint64_t seed, int64_t n_chunks,
+                                        const int64_t *host_chunk_off, const int32_t *host_chunk_task);
+
 /* One CoCoA round (Sec. 2.1 Eq. 1, Eq. 2 and worker structure with L = 1; Sec. 5.1: SCD local solver, sigma =
  * number of tasks). Each partition draws this round's seeded visiting order (members ordered by
  * mix64(mix64(seed ^ 0xD1B54A32D192ED03) ^ mix64(round * 2^32 + epoch) ^ id)), walks it strictly in order for H

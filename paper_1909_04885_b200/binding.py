@@ -24,7 +24,8 @@ MEM_HOST, MEM_DEVICE = 0, 1
 EXPORTED = ["chicle_glm_create", "chicle_partition", "chicle_cocoa_round", "chicle_duality_gap", "chicle_get_alpha",
             "chicle_get_v", "chicle_get_partition", "chicle_get_permutation", "chicle_set_state", "chicle_get_info",
             "chicle_last_error", "chicle_glm_destroy", "chicle_partition_noalloc", "chicle_partition_sizes",
-            "chicle_cocoa_round_steps"]
+            "chicle_cocoa_round_steps", "chicle_chunks_cut", "chicle_chunks_assign", "chicle_chunks_scale_in",
+            "chicle_chunks_scale_out", "chicle_chunks_rebalance_step", "chicle_partition_chunks"]
 
 
 class ChicleError(RuntimeError):
@@ -74,6 +75,18 @@ def load():
     lib.chicle_cocoa_round.argtypes = [vp, i64, f32, C.POINTER(RoundStats)]
     lib.chicle_cocoa_round_steps.restype = C.c_int
     lib.chicle_cocoa_round_steps.argtypes = [vp, vp, f32, C.POINTER(RoundStats)]
+    lib.chicle_chunks_cut.restype = i64
+    lib.chicle_chunks_cut.argtypes = [i64, vp, i64, i64, vp]
+    lib.chicle_chunks_assign.restype = C.c_int
+    lib.chicle_chunks_assign.argtypes = [i64, i32, C.c_uint64, vp]
+    lib.chicle_chunks_scale_in.restype = C.c_int
+    lib.chicle_chunks_scale_in.argtypes = [i64, i32, i32, vp]
+    lib.chicle_chunks_scale_out.restype = C.c_int
+    lib.chicle_chunks_scale_out.argtypes = [i64, i32, i32, C.c_uint64, vp]
+    lib.chicle_chunks_rebalance_step.restype = C.c_int
+    lib.chicle_chunks_rebalance_step.argtypes = [i64, vp, i32, vp, vp]
+    lib.chicle_partition_chunks.restype = C.c_int
+    lib.chicle_partition_chunks.argtypes = [vp, i32, C.c_uint64, i64, vp, vp]
     lib.chicle_duality_gap.restype = C.c_int
     lib.chicle_duality_gap.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     for name in ("chicle_get_alpha", "chicle_get_v"):
@@ -220,6 +233,15 @@ class Glm:
             self._check(self._lib.chicle_partition_sizes(self._h, K, C.c_uint64(seed & (2**64 - 1)), _ptr(sz)))
         self.K = K
 
+    def partition_chunks(self, K: int, seed: int, chunk_off, chunk_task):
+        """``chicle_partition_chunks``: the partition that a placement of data chunks on K tasks induces."""
+        off = np.ascontiguousarray(chunk_off, np.int64)
+        task = np.ascontiguousarray(chunk_task, np.int32)
+        if off.size != task.size + 1:
+            raise ValueError("chunk_off must have one entry more than chunk_task")
+        self._check(self._lib.chicle_partition_chunks(self._h, K, C.c_uint64(seed & (2**64 - 1)), task.size, _ptr(off), _ptr(task)))
+        self.K = K
+
     def cocoa_round(self, H: int = 0, sigma_prime: Optional[float] = None, stats: bool = False, steps=None):
         """One round; ``steps`` (K integers, 0 <= steps[k] <= size of partition k) gives each partition its own budget."""
         sp = float(self.K if sigma_prime is None else sigma_prime)
@@ -303,3 +325,51 @@ def partition_noalloc(n_coord: int, K: int, seed: int, owner_out, members_out, d
                                       C.c_void_p(owner_out.data_ptr()), C.c_void_p(members_out.data_ptr()), buf, 256)
     if st != OK:
         raise ChicleError(st, buf.value.decode())
+
+
+# ---- mobile data chunks: host-side placement logic of the library (argument marshalling only) -------------------
+def chunks_cut(n_coord: int, chunk_bytes: int, indptr=None, dense_dim: int = 0) -> np.ndarray:
+    """``chicle_chunks_cut``: chunk offsets for chunks of at most ``chunk_bytes``."""
+    off = np.empty(n_coord + 1, np.int64)
+    ip = None if indptr is None else np.ascontiguousarray(indptr, np.int64)
+    c = load().chicle_chunks_cut(n_coord, None if ip is None else _ptr(ip), dense_dim, chunk_bytes, _ptr(off))
+    if c < 0:
+        raise ValueError("chicle_chunks_cut: bad arguments")
+    return off[:c + 1].copy()
+
+
+def chunks_assign(n_chunks: int, K: int, seed: int) -> np.ndarray:
+    task = np.empty(n_chunks, np.int32)
+    st = load().chicle_chunks_assign(n_chunks, K, C.c_uint64(seed & (2**64 - 1)), _ptr(task))
+    if st != OK:
+        raise ChicleError(st, "chicle_chunks_assign: need 1 <= K <= number of chunks")
+    return task
+
+
+def chunks_scale_in(task, K_old: int, K_new: int) -> np.ndarray:
+    out = np.array(task, np.int32, copy=True)
+    st = load().chicle_chunks_scale_in(out.size, K_old, K_new, _ptr(out))
+    if st != OK:
+        raise ChicleError(st, "chicle_chunks_scale_in: need 1 <= K_new <= K_old")
+    return out
+
+
+def chunks_scale_out(task, K_old: int, K_new: int, seed: int) -> np.ndarray:
+    out = np.array(task, np.int32, copy=True)
+    st = load().chicle_chunks_scale_out(out.size, K_old, K_new, C.c_uint64(seed & (2**64 - 1)), _ptr(out))
+    if st != OK:
+        raise ChicleError(st, "chicle_chunks_scale_out: need 1 <= K_old <= K_new and tasks in [0, K_old)")
+    return out
+
+
+def chunks_rebalance_step(task, chunk_off, K: int, time_per_sample):
+    """Returns (new placement, whether a chunk moved)."""
+    out = np.array(task, np.int32, copy=True)
+    off = np.ascontiguousarray(chunk_off, np.int64)
+    t = np.ascontiguousarray(time_per_sample, np.float64)
+    if off.size != out.size + 1 or t.size != K:
+        raise ValueError("chunk_off needs one entry more than task, time_per_sample K entries")
+    r = load().chicle_chunks_rebalance_step(out.size, _ptr(off), K, _ptr(t), _ptr(out))
+    if r < 0:
+        raise ValueError("chicle_chunks_rebalance_step: bad arguments")
+    return out, bool(r)

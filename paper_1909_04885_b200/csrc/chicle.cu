@@ -271,10 +271,32 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
     return CHICLE_OK;
 }
 
-static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed, const int64_t *sizes)
+// A placement of data chunks on tasks (host arrays): chunk c holds coordinates off[c] .. off[c + 1] - 1.
+struct ChunkPlacement {
+    int64_t C;
+    const int64_t *off;
+    const int32_t *task;
+};
+
+static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed, const int64_t *sizes, const ChunkPlacement *chunks = nullptr)
 {
     if (!h) return CHICLE_ERR_INVALID_ARG;
     if (K < 1 || (int64_t)K > h->n_coord) return fail(h, CHICLE_ERR_INVALID_ARG, "need 1 <= K <= number of coordinates");
+    std::vector<int64_t> chunk_sizes;
+    if (chunks) {
+        const int64_t C = chunks->C;
+        if (C < K || C > h->n_coord || !chunks->off || !chunks->task || chunks->off[0] != 0 || chunks->off[C] != h->n_coord)
+            return fail(h, CHICLE_ERR_INVALID_ARG, "chunk offsets must run from 0 to the number of coordinates, with K <= chunks <= coordinates");
+        chunk_sizes.assign((size_t)K, 0);
+        for (int64_t c = 0; c < C; ++c) {
+            if (chunks->off[c + 1] <= chunks->off[c]) return fail(h, CHICLE_ERR_INVALID_ARG, "chunk offsets must increase strictly");
+            if (chunks->task[c] < 0 || chunks->task[c] >= K) return fail(h, CHICLE_ERR_INVALID_ARG, "a chunk's task must lie in [0, K)");
+            chunk_sizes[(size_t)chunks->task[c]] += chunks->off[c + 1] - chunks->off[c];
+        }
+        for (int32_t k = 0; k < K; ++k)
+            if (chunk_sizes[(size_t)k] == 0) return fail(h, CHICLE_ERR_INVALID_ARG, "every task must hold at least one chunk");
+        sizes = chunk_sizes.data();
+    }
     if (sizes) {
         int64_t tot = 0;
         for (int32_t k = 0; k < K; ++k) {
@@ -364,10 +386,29 @@ static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed,
     h->seed = seed;
     e = cudaMemcpyAsync(part_off, h_off, ((size_t)K + 1) * 8, cudaMemcpyHostToDevice, h->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(U, 0, (size_t)K * (size_t)h->dim * 4, h->stream);
-    if (e == cudaSuccess) e = launch_partition(*h, K, seed);
+    int64_t *d_coff = nullptr;
+    int32_t *d_ctask = nullptr;
+    if (chunks && e == cudaSuccess) {
+        // the placement travels as two temporary device arrays, released once the kernels that read them are done
+        if (!alloc_into(h, d_coff, (size_t)chunks->C + 1) || !alloc_into(h, d_ctask, (size_t)chunks->C)) {
+            dev_free(h, d_coff);
+            h->K = 0;
+            return fail(h, CHICLE_ERR_OOM, "device allocation failed (chunk placement)");
+        }
+        e = cudaMemcpyAsync(d_coff, chunks->off, ((size_t)chunks->C + 1) * 8, cudaMemcpyHostToDevice, h->stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(d_ctask, chunks->task, (size_t)chunks->C * 4, cudaMemcpyHostToDevice, h->stream);
+        if (e == cudaSuccess) e = launch_partition_chunks(*h, K, chunks->C, d_coff, d_ctask);
+    } else if (e == cudaSuccess) {
+        e = launch_partition(*h, K, seed);
+    }
     // the host copy of part_off is reused by later calls, so finish the upload before returning
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
-    if (e != cudaSuccess) return fail_cuda(h, e, "partition kernels");
+    if (d_coff) dev_free(h, d_coff);
+    if (d_ctask) dev_free(h, d_ctask);
+    if (e != cudaSuccess) {
+        h->K = 0; // the partition map is not valid: a new partition call is required
+        return fail_cuda(h, e, "partition kernels");
+    }
     return CHICLE_OK;
 }
 
@@ -377,6 +418,14 @@ chicle_status_t chicle_partition_sizes(chicle_glm_t *h, int32_t K, uint64_t seed
 {
     if (h && !host_sizes) return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_partition_sizes: sizes is NULL");
     return partition_impl(h, K, seed, host_sizes);
+}
+
+chicle_status_t chicle_partition_chunks(chicle_glm_t *h, int32_t K, uint64_t seed, int64_t n_chunks, const int64_t *host_chunk_off,
+                                        const int32_t *host_chunk_task)
+{
+    if (!h) return CHICLE_ERR_INVALID_ARG;
+    const ChunkPlacement cp{n_chunks, host_chunk_off, host_chunk_task};
+    return partition_impl(h, K, seed, nullptr, &cp);
 }
 
 // One round. host_steps == nullptr: every partition takes H steps (0: one local epoch). Otherwise partition k takes

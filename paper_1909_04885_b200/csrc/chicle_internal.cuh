@@ -126,6 +126,7 @@ struct Glm {
 cudaError_t launch_validate(Glm &g);
 cudaError_t launch_sqnorm(Glm &g);
 cudaError_t launch_partition(Glm &g, int32_t K, uint64_t seed);           // fills owner, members
+cudaError_t launch_partition_chunks(Glm &g, int32_t K, int64_t C, const int64_t *chunk_off, const int32_t *chunk_task); // device arrays
 cudaError_t launch_permutation(Glm &g, int64_t round, int64_t epochs);    // fills perm[epochs * n_coord]
 cudaError_t launch_local_solver(Glm &g, int64_t H, float sigma_prime, int *variant);
 cudaError_t launch_reduce(Glm &g);                                        // v += sum_k U_k ; U = 0 ; resid

@@ -142,6 +142,35 @@ cudaError_t launch_partition(Glm &g, int32_t K, uint64_t seed)
     return cudaGetLastError();
 }
 
+// owner[i] = task of the chunk that holds coordinate i: chunk_off[c] <= i < chunk_off[c + 1]
+__global__ void k_owner_from_chunks(int64_t n, int64_t C, const int64_t *__restrict__ chunk_off,
+                                    const int32_t *__restrict__ chunk_task, int32_t *__restrict__ owner)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) {
+        int64_t lo = 0, hi = C;
+        while (hi - lo > 1) {
+            const int64_t mid = (lo + hi) >> 1;
+            if (chunk_off[mid] <= i) lo = mid;
+            else hi = mid;
+        }
+        owner[i] = chunk_task[lo];
+    }
+}
+
+cudaError_t launch_partition_chunks(Glm &g, int32_t K, int64_t C, const int64_t *chunk_off, const int32_t *chunk_task)
+{
+    const int64_t n = g.n_coord;
+    SortWorkspace &w = g.sortws;
+    const int T = 256;
+    k_owner_from_chunks<<<blocks_for(n, T), T, 0, g.stream>>>(n, C, chunk_off, chunk_task, g.owner);
+    // members: ids 0..n-1 (ascending) stably grouped by owner
+    k_iota<<<blocks_for(n, T), T, 0, g.stream>>>(n, w.vals[0]);
+    cudaError_t e = owner_passes(g, K, w.vals[0], reinterpret_cast<int32_t *>(w.keys[0]), g.members);
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_permutation(Glm &g, int64_t round, int64_t epochs)
 {
     const int64_t n = g.n_coord;

@@ -136,3 +136,139 @@ def test_rounds_on_a_chunk_partition_keep_the_invariants():
         prev = g["dual"]
         v2 = o.recompute_shared_vector()
         assert np.abs(v2 - o.v).max() <= 1e-12 * max(1.0, np.abs(v2).max())
+
+
+# ------------------------------------------------------------------ the library's host functions against the oracle
+def _lib():
+    from paper_1909_04885_b200 import binding, build
+    build.build()
+    return binding
+
+
+def test_library_chunk_functions_match_the_oracle_bit_for_bit():
+    oracle.build()
+    b = _lib()
+    rng = np.random.default_rng(3)
+    for n, bytes_ in ((1, 64), (50, 8), (5000, 4096), (5000, 300)):
+        nnz = rng.poisson(6, n)
+        nnz[rng.integers(0, n, max(1, n // 50))] = 400  # a few coordinates larger than a chunk
+        indptr = np.concatenate([[0], np.cumsum(nnz)]).astype(np.int64)
+        assert np.array_equal(b.chunks_cut(n, bytes_, indptr), och.cut(n, bytes_, indptr))
+    assert np.array_equal(b.chunks_cut(1000, 1000, None, 28), och.cut(1000, 1000, None, 28))
+    for C, K, seed in ((1, 1, 0), (17, 17, 1), (1000, 7, 2**63 + 5), (4097, 64, 3)):
+        assert np.array_equal(b.chunks_assign(C, K, seed), och.assign(C, K, seed))
+    t = och.assign(1500, 24, 4)
+    for K_new in (24, 23, 5, 1):
+        assert np.array_equal(b.chunks_scale_in(t, 24, K_new), och.scale_in(t, 24, K_new))
+    t = och.assign(1500, 3, 5)
+    for K_new, seed in ((3, 0), (4, 1), (16, 2), (100, 2**64 - 1)):
+        assert np.array_equal(b.chunks_scale_out(t, 3, K_new, seed), och.scale_out(t, 3, K_new, seed))
+    # rebalancing: the same sequence of moves until both stop
+    off = och.cut(5000, 300, indptr)
+    C = len(off) - 1
+    K = 5
+    speed = [1.0, 2.5, 1.0, 0.7, 1.2]
+    to, tl = och.assign(C, K, 0), b.chunks_assign(C, K, 0)
+    ln = np.diff(off)
+    for it in range(10 * C):
+        to, mo = och.rebalance_step(to, ln, K, speed)
+        tl, ml = b.chunks_rebalance_step(tl, off, K, speed)
+        assert mo == ml and np.array_equal(to, tl)
+        if not mo:
+            break
+    assert it > 3 and not mo
+
+
+def test_library_chunk_functions_refuse_bad_arguments():
+    b = _lib()
+    with pytest.raises(b.ChicleError):
+        b.chunks_assign(4, 5, 0)
+    with pytest.raises(b.ChicleError):
+        b.chunks_scale_in(np.zeros(4, np.int32), 2, 3)
+    with pytest.raises(b.ChicleError):
+        b.chunks_scale_out(np.zeros(4, np.int32), 3, 2, 0)
+    with pytest.raises(b.ChicleError):
+        b.chunks_scale_out(np.array([0, 5], np.int32), 2, 4, 0)
+    with pytest.raises(ValueError):
+        b.chunks_cut(0, 64, np.zeros(1, np.int64))
+
+
+# ------------------------------------------------------------------ on the GPU: partitions from placements, rounds
+@pytest.mark.gpu
+def test_chunk_partitions_and_elastic_rounds_match_the_oracle():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    b = _lib()
+    from paper_1909_04885_b200 import datagen
+    from parity_util import REL_TOL, gap_close, make_pair, rel_l2
+    w = datagen.make("hinge_csr", 100)
+    orc, glm = make_pair(w)
+    try:
+        off = b.chunks_cut(w.n_coord, 16384, w.indptr)
+        assert np.array_equal(off, och.cut(w.n_coord, 16384, w.indptr))
+        C = len(off) - 1
+        task = b.chunks_assign(C, 16, 1)
+        schedule = [(16, None), (16, None), (6, "in"), (6, None), (24, "out"), (24, "rebalance"), (24, None)]
+        K_prev = 16
+        for r, (K, move) in enumerate(schedule):
+            if move == "in":
+                task = b.chunks_scale_in(task, K_prev, K)
+            elif move == "out":
+                task = b.chunks_scale_out(task, K_prev, K, 7)
+            elif move == "rebalance":
+                speed = [1.0 + (k % 3) for k in range(K)]
+                for _ in range(40):
+                    task, moved = b.chunks_rebalance_step(task, off, K, speed)
+                    assert moved
+            K_prev = K
+            orc.partition_chunks(K, 3, off, task)
+            glm.partition_chunks(K, 3, off, task)
+            assert np.array_equal(glm.get_partition(), orc.owner)
+            for k in (0, K // 2, K - 1):
+                n_k = int(orc.part_off[k + 1] - orc.part_off[k])
+                assert np.array_equal(glm.get_permutation(r, k, n_k), orc.permutation(r, k))
+            orc.cocoa_round(0, float(K))
+            glm.cocoa_round(0, float(K))
+            assert rel_l2(glm.get_alpha(), orc.state) <= REL_TOL and rel_l2(glm.get_v(), orc.v) <= REL_TOL
+            ok, tol = gap_close(glm.duality_gap(), orc.duality_gap())
+            assert ok
+        # bad placements leave the handle as it was
+        before = glm.get_partition().copy()
+        for bad_off, bad_task in ((off[:-1], task[:-1]), (off, np.where(task == 3, 4, task)), (off, task + 1)):
+            with pytest.raises(b.ChicleError) as e:
+                glm.partition_chunks(24, 3, bad_off, bad_task)
+            assert e.value.status == 1
+        assert np.array_equal(before, glm.get_partition())
+        glm.cocoa_round(0, 24.0)
+    finally:
+        glm.close()
+
+
+@pytest.mark.gpu
+def test_chunk_partition_dense_and_one_chunk_per_coordinate():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    b = _lib()
+    from paper_1909_04885_b200 import datagen
+    from parity_util import REL_TOL, make_pair, rel_l2
+    w = datagen.make("hinge_dense", 64)
+    orc, glm = make_pair(w)
+    try:
+        n = w.n_coord
+        # one chunk per coordinate with the random deal is chicle_partition itself
+        off = np.arange(n + 1, dtype=np.int64)
+        glm.partition_chunks(5, 9, off, b.chunks_assign(n, 5, 9))
+        a = glm.get_partition().copy()
+        glm.partition(5, 9)
+        assert np.array_equal(a, glm.get_partition())
+        off = b.chunks_cut(n, 40 * (4 * w.n_cols + 8), None, w.n_cols)
+        task = b.chunks_assign(len(off) - 1, 4, 2)
+        for K, t in ((4, task), (2, b.chunks_scale_in(task, 4, 2))):
+            orc.partition_chunks(K, 1, off, t)
+            glm.partition_chunks(K, 1, off, t)
+            assert np.array_equal(glm.get_partition(), orc.owner)
+            orc.cocoa_round(0, float(K))
+            glm.cocoa_round(0, float(K))
+            assert rel_l2(glm.get_alpha(), orc.state) <= REL_TOL and rel_l2(glm.get_v(), orc.v) <= REL_TOL
+    finally:
+        glm.close()
