@@ -18,6 +18,7 @@
 // Every wait is bounded; when one runs out the kernel records it in the status word and all roles return.
 #include <cstdlib>
 #include <cstring>
+#include <vector>
 
 #include "solver_common.cuh"
 
@@ -396,9 +397,40 @@ cudaError_t launch_local_solver(Glm &g, int64_t H, float sigma_prime, int *varia
     const char *force = getenv("CHICLE_FORCE_VARIANT"); // debugging aid: "ring" selects the unblocked solver
     const bool ring = force && strcmp(force, "ring") == 0;
     const bool blocked = force && strcmp(force, "blocked") == 0;
-    if (g.la_rec && !P.multi_epoch && !ring && !blocked && (!dense || g.dim <= lookahead_max_dense_dim())) {
+    if (g.la_rec && !ring && !blocked && (!dense || g.dim <= lookahead_max_dense_dim())) {
         *variant = dense ? 5 : 4;
-        return launch_lookahead_solver(g, P);
+        if (!P.multi_epoch) return launch_lookahead_solver(g, P);
+        // H spans several local epochs: one prepare + chain pair per epoch. Partition k takes what is left of its H
+        // steps, at most one pass over its coordinates, along that epoch's visiting order; the prepared headers of an
+        // epoch see the state the epoch before left, and the accumulated updates carry over in U.
+        const int64_t epochs = (H + min_nk - 1) / min_nk;
+        std::vector<int64_t> steps((size_t)g.K);
+        P.multi_epoch = 0;
+        P.H = 0;
+        P.steps_k = g.d_steps;
+        const bool time_prepare = g.time_prepare;
+        cudaError_t e = cudaSuccess;
+        for (int64_t ep = 0; ep < epochs && e == cudaSuccess; ++ep) {
+            int64_t total = 0;
+            for (int32_t k = 0; k < g.K; ++k) {
+                const int64_t nk = g.h_part_off[k + 1] - g.h_part_off[k];
+                const int64_t left = H - ep * nk;
+                steps[(size_t)k] = left <= 0 ? 0 : (left < nk ? left : nk);
+                total += steps[(size_t)k];
+            }
+            if (total == 0) break;
+            // a pageable source: the runtime has taken its copy when the call returns, and the copy is ordered behind
+            // the kernels of the epoch before on the stream
+            e = cudaMemcpyAsync(g.d_steps, steps.data(), (size_t)g.K * sizeof(int64_t), cudaMemcpyHostToDevice, g.stream);
+            if (e != cudaSuccess) break;
+            P.perm = g.perm + (size_t)ep * (size_t)g.n_coord;
+            g.round_steps = steps.data();
+            g.time_prepare = time_prepare && ep == 0; // the prepare time reported is the first epoch's
+            e = launch_lookahead_solver(g, P);
+        }
+        g.round_steps = nullptr;
+        g.time_prepare = time_prepare;
+        return e;
     }
     if (dense && g.dim <= blocked_solver_max_dense_dim() && !ring) {
         *variant = 3;

@@ -126,6 +126,29 @@ def test_partial_and_multi_epoch_H(H):
     run_parity(tiny_csr(100, 30, seed=5, K=4), H=H)
 
 
+def test_rounds_of_several_local_epochs(monkeypatch):
+    # H beyond one local epoch: the look-ahead solver runs once per epoch; ragged last epoch, unequal partitions
+    # (the small ones go round more often), all three losses; then the blocked solver's own multi-epoch walk
+    w = datagen.make("hinge_csr", 100)
+    n_k = w.n_coord // w.phases[0].K
+    run_parity(w, rounds=3, H=2 * n_k + n_k // 3)
+    run_parity(w, rounds=2, H=n_k + 1)
+    run_parity(tiny_csr(400, 40, seed=8, K=3), H=700, sizes=[50, 300, 50])
+    run_parity(tiny_dense(500, 28, seed=2, loss="logistic", K=4), H=300)
+    w = datagen.make("ridge_csc", 100)
+    w.phases = [Phase(0, 4, 1, 4.0)]
+    run_parity(w, rounds=2, H=w.n_coord // 4 * 2 + 17)
+    glm = binding.from_workload(tiny_csr(400, 40, seed=8, K=4))
+    try:
+        glm.partition(4, 0)
+        st = glm.cocoa_round(250, 4.0, stats=True)
+        assert st["solver_variant"] == 4 and st["steps"] == 1000
+    finally:
+        glm.close()
+    monkeypatch.setenv("CHICLE_FORCE_VARIANT", "blocked")
+    run_parity(tiny_csr(400, 40, seed=8, K=3), H=700, sizes=[50, 300, 50])
+
+
 def test_ridge_small_with_long_and_empty_columns():
     rng = np.random.default_rng(11)
     n, d = 300, 500
@@ -285,7 +308,7 @@ def test_older_solvers_still_match(variant, monkeypatch):
     run_parity(tiny_dense(500, 28, seed=2, loss="logistic", K=4))
 
 
-def test_lookahead_solver_is_the_default_for_single_epoch_rounds():
+def test_lookahead_solver_is_the_default():
     for w, want in ((datagen.make("hinge_csr", 100), 4), (datagen.make("hinge_dense", 4), 5)):
         glm = binding.from_workload(w)
         try:
@@ -293,7 +316,7 @@ def test_lookahead_solver_is_the_default_for_single_epoch_rounds():
             assert glm.cocoa_round(0, float(w.phases[0].K), stats=True)["solver_variant"] == want
             assert glm.cocoa_round(5, float(w.phases[0].K), stats=True)["solver_variant"] == want
             n_k = w.n_coord // w.phases[0].K
-            assert glm.cocoa_round(2 * n_k, float(w.phases[0].K), stats=True)["solver_variant"] in (1, 3)
+            assert glm.cocoa_round(2 * n_k, float(w.phases[0].K), stats=True)["solver_variant"] == want  # once per local epoch
         finally:
             glm.close()
 
