@@ -87,8 +87,10 @@ typedef struct {
     int64_t steps;        /* coordinate steps taken in this round, all partitions               */
     int32_t solver_variant; /* 0 dense ring, 1 sparse blocked, 2 sparse ring, 3 dense blocked (rows <= 128),
                                4 sparse look-ahead, 5 dense look-ahead (rows <= 128) */
-    float ms_prepare;     /* part of ms_local spent in the look-ahead solver's prepare kernel (variants 4, 5; when H
-                             spans several local epochs: the first epoch's), else 0 */
+    float ms_prepare;     /* part of ms_local before the look-ahead solver's first chain launch starts (variants 4, 5):
+                             the prepare kernel of the whole round, or of its first slice when a long round is cut
+                             into slices whose prepare kernels run beside the chain kernels; when H spans several
+                             local epochs: the first epoch's; else 0 */
 } chicle_round_stats_t;
 
 /* Create a training problem (Sec. 2.2, Sec. 5.1: a GLM trained by CoCoA with a local SCD solver; Sec. 4.4:

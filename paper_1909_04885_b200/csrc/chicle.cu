@@ -96,6 +96,12 @@ void destroy_impl(chicle_glm *h)
     if (!h) return;
     (void)cudaSetDevice(h->device);
     (void)cudaStreamSynchronize(h->stream);
+    if (h->la_stream) {
+        (void)cudaStreamSynchronize(h->la_stream);
+        (void)cudaStreamDestroy(h->la_stream);
+    }
+    for (auto &ev : h->la_ev)
+        if (ev) (void)cudaEventDestroy(ev);
     while (!h->owned.empty()) dev_free(h, h->owned.back());
     if (h->h_status) (void)cudaFreeHost(h->h_status);
     if (h->h_gap) (void)cudaFreeHost(h->h_gap);
@@ -192,6 +198,16 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
         return bail(CHICLE_ERR_OOM, "pinned host allocation failed");
     for (auto &ev : h->ev)
         if ((e = cudaEventCreate(&ev)) != cudaSuccess) return bail_cuda(e, "cudaEventCreate");
+    {
+        // the look-ahead solver's side stream: lowest priority, so that the chain kernels get their SMs first, and
+        // non-blocking, so that it does not order itself against the legacy default stream
+        int least = 0, greatest = 0;
+        (void)cudaDeviceGetStreamPriorityRange(&least, &greatest);
+        if ((e = cudaStreamCreateWithPriority(&h->la_stream, cudaStreamNonBlocking, least)) != cudaSuccess)
+            return bail_cuda(e, "cudaStreamCreateWithPriority");
+        for (auto &ev : h->la_ev)
+            if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return bail_cuda(e, "cudaEventCreate");
+    }
 
     cudaStream_t s = h->stream;
     if (dense) {
@@ -354,22 +370,23 @@ static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed,
         delete[] h->h_part_off;
         U = newU; part_off = new_off; h_off = new_hoff;
         // the look-ahead solver's per-round records (their number depends on K); without them the blocked solver runs
-        dev_free(h, h->la_rec); dev_free(h, h->la_dir); dev_free(h, h->la_cursor); dev_free(h, h->la_blk_base);
-        h->la_rec = nullptr; h->la_dir = nullptr; h->la_cursor = nullptr; h->la_blk_base = nullptr; h->la_rec_bytes = 0;
+        dev_free(h, h->la_rec); dev_free(h, h->la_dir); dev_free(h, h->la_cursor); dev_free(h, h->la_blk_base); dev_free(h, h->la_slice);
+        h->la_rec = nullptr; h->la_dir = nullptr; h->la_cursor = nullptr; h->la_blk_base = nullptr; h->la_slice = nullptr; h->la_rec_bytes = 0;
         const bool dense_fmt = h->fmt == CHICLE_FMT_DENSE_ROWMAJOR;
         if (!dense_fmt || h->dim <= lookahead_max_dense_dim()) {
             size_t rec_bytes = 0, dir_bytes = 0;
             lookahead_workspace(n, h->nnz, K, dense_fmt, h->dim, &rec_bytes, &dir_bytes);
             unsigned char *rec = nullptr, *dir = nullptr;
             if (alloc_into(h, rec, rec_bytes) && alloc_into(h, dir, dir_bytes) && alloc_into(h, h->la_cursor, 32) &&
-                alloc_into(h, h->la_blk_base, (size_t)K + 1)) {
+                alloc_into(h, h->la_blk_base, (size_t)lookahead_max_slices() * ((size_t)K + 1)) &&
+                alloc_into(h, h->la_slice, (size_t)lookahead_max_slices() * 2 * (size_t)K)) {
                 h->la_rec = rec;
                 h->la_dir = dir;
                 h->la_rec_bytes = rec_bytes;
                 (void)cudaMemsetAsync(h->la_cursor, 0, 32 * sizeof(unsigned long long), h->stream);
             } else {
-                dev_free(h, rec); dev_free(h, dir); dev_free(h, h->la_cursor); dev_free(h, h->la_blk_base);
-                h->la_cursor = nullptr; h->la_blk_base = nullptr;
+                dev_free(h, rec); dev_free(h, dir); dev_free(h, h->la_cursor); dev_free(h, h->la_blk_base); dev_free(h, h->la_slice);
+                h->la_cursor = nullptr; h->la_blk_base = nullptr; h->la_slice = nullptr;
             }
         }
     }

@@ -104,7 +104,10 @@ struct Glm {
     void *la_dir = nullptr;
     unsigned long long *la_cursor = nullptr;
     size_t la_rec_bytes = 0;
-    int64_t *la_blk_base = nullptr; // K+1: first block of each partition in this round's numbering of the blocks
+    int64_t *la_blk_base = nullptr; // per slice K+1: first block of each partition in the slice's numbering of the blocks
+    int64_t *la_slice = nullptr;    // per slice 2K: every partition's step count and first step in that slice
+    cudaStream_t la_stream = nullptr; // side stream (lowest priority) for the later slices' prepare kernels
+    cudaEvent_t la_ev[3] = {nullptr, nullptr, nullptr}; // slice s is prepared
     bool time_prepare = false; // record ev[4] between the prepare and the chain kernel (round statistics asked for)
 
     SortWorkspace sortws;
@@ -139,6 +142,7 @@ cudaError_t launch_gather_f32(Glm &g, const float *src, const int32_t *map, int6
 cudaError_t launch_lookahead_solver(Glm &g, const struct SolverParams &P);
 void lookahead_workspace(int64_t n_coord, int64_t nnz, int32_t K, bool dense, int64_t dim, size_t *rec_bytes, size_t *dir_bytes);
 int lookahead_max_dense_dim();
+int lookahead_max_slices();
 int blocked_solver_hot_ids();
 int blocked_solver_short_cap();
 

@@ -37,6 +37,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <vector>
 
 #include "solver_common.cuh"
 
@@ -254,8 +255,8 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) k_lookahead_prepare(c
     int k;
     int64_t b;
     block_to_part(P, bid, k, b);
-    const int64_t off = P.S.part_off[k];
-    const int64_t nk = P.S.part_off[k + 1] - off;
+    const int64_t nk = P.S.part_off[k + 1] - P.S.part_off[k];
+    const int64_t off = P.S.part_off[k] + (P.S.first_k ? P.S.first_k[k] : 0); // of this launch's first step in the order
     const int64_t steps = steps_of(P, k, nk);
     const int cnt = (int)((steps - b * kLB) < kLB ? (steps - b * kLB) : kLB);
 #ifdef CHICLE_LA_TIMING
@@ -497,8 +498,8 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
     int k;
     int64_t b;
     block_to_part(P, bid, k, b);
-    const int64_t off = P.S.part_off[k];
-    const int64_t nk = P.S.part_off[k + 1] - off;
+    const int64_t nk = P.S.part_off[k + 1] - P.S.part_off[k];
+    const int64_t off = P.S.part_off[k] + (P.S.first_k ? P.S.first_k[k] : 0); // of this launch's first step in the order
     const int64_t steps = steps_of(P, k, nk);
     const int cnt = (int)((steps - b * kLB) < kLB ? (steps - b * kLB) : kLB);
     const int dim = (int)P.S.dim;
@@ -990,37 +991,34 @@ template <int LOSS, bool DENSE, int HOT, int TMAX, int NCH> cudaError_t launch_c
     return e;
 }
 
-template <int LOSS, int NZ, int HT, int THREADS> cudaError_t launch_prepare(Glm &g, const LookParams &P, unsigned nb)
+template <int LOSS, int NZ, int HT, int THREADS> cudaError_t launch_prepare(Glm &g, const LookParams &P, unsigned nb, cudaStream_t stream)
 {
+    (void)g;
     using Shared = PreShared<NZ, HT, THREADS>;
     auto pre = k_lookahead_prepare<LOSS, NZ, HT, THREADS>;
     cudaError_t e = cudaFuncSetAttribute(pre, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Shared));
     if (e != cudaSuccess) return e;
-    pre<<<nb, THREADS, sizeof(Shared), g.stream>>>(P);
+    pre<<<nb, THREADS, sizeof(Shared), stream>>>(P);
     return cudaGetLastError();
 }
 
-template <int LOSS> cudaError_t launch_loss(Glm &g, LookParams &P)
+// The prepare kernel of one launch's blocks on `stream`.
+template <int LOSS> cudaError_t launch_prepare_on(Glm &g, const LookParams &P, cudaStream_t stream)
 {
     const unsigned nb = (unsigned)P.n_blocks;
-    cudaError_t e = cudaMemsetAsync(P.cursor, 0, sizeof(unsigned long long), g.stream);
-    if (e != cudaSuccess) return e;
     if (g.fmt == CHICLE_FMT_DENSE_ROWMAJOR) {
-        k_lookahead_prepare_dense<LOSS><<<nb, kPreThreads, 0, g.stream>>>(P);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-        if (g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
-        return launch_chain<LOSS, true, kCapL, 4, 4>(g, P);
+        k_lookahead_prepare_dense<LOSS><<<nb, kPreThreads, 0, stream>>>(P);
+        return cudaGetLastError();
     }
     // blocks of up to 2 048 non-zeros (32 coordinates of 50 on average, with room): the small variant, four CTAs per SM
     const double avg_block = 32.0 * (double)g.nnz / (double)g.n_coord;
-    if (avg_block * 1.25 <= 2048.0) e = launch_prepare<LOSS, 2048, 2048, 256>(g, P, nb);
-    else e = launch_prepare<LOSS, kMaxNz, kHT, kPreThreadsS>(g, P, nb);
-    if (e != cudaSuccess) return e;
+    cudaError_t e;
+    if (avg_block * 1.25 <= 2048.0) e = launch_prepare<LOSS, 2048, 2048, 256>(g, P, nb, stream);
+    else e = launch_prepare<LOSS, kMaxNz, kHT, kPreThreadsS>(g, P, nb, stream);
 #ifdef CHICLE_LA_TIMING
-    {
+    if (e == cudaSuccess) {
         unsigned long long t[8] = {0};
-        (void)cudaStreamSynchronize(g.stream);
+        (void)cudaStreamSynchronize(stream);
         (void)cudaMemcpy(t, P.cursor + 16, sizeof(t), cudaMemcpyDeviceToHost);
         (void)cudaMemset(P.cursor + 16, 0, sizeof(t));
         fprintf(stderr, "lookahead prepare, cycles per CTA: headers %.0f insert %.0f count %.0f place %.0f number %.0f entries %.0f gram %.0f write %.0f\n",
@@ -1028,46 +1026,136 @@ template <int LOSS> cudaError_t launch_loss(Glm &g, LookParams &P)
                 t[6] / (double)nb, t[7] / (double)nb);
     }
 #endif
-    if (g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
+    return e;
+}
+
+// The chain kernel over the blocks that a prepare launch with the same parameters made (on the handle's stream).
+template <int LOSS> cudaError_t launch_chain_on(Glm &g, const LookParams &P)
+{
+    if (g.fmt == CHICLE_FMT_DENSE_ROWMAJOR) return launch_chain<LOSS, true, kCapL, 4, 4>(g, P);
     if (g.hot_variant) return launch_chain<LOSS, false, kHotSkew, kTmax, 2>(g, P);
     return launch_chain<LOSS, false, 4, kTmax, 4>(g, P);
+}
+
+// A round's launches. One slice: prepare, then chain. Several slices (consecutive pieces of every partition's walk):
+// the first slice's prepare on the handle's stream; the later slices' prepares on the side stream, behind the first
+// one, so that they fill the SMs the chain kernels leave idle; every chain launch waits for its slice's prepare.
+template <int LOSS> cudaError_t launch_slices(Glm &g, const LookParams *P, int n_slices)
+{
+    cudaError_t e = launch_prepare_on<LOSS>(g, P[0], g.stream);
+    if (e != cudaSuccess) return e;
+    if (g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
+    if (n_slices > 1) {
+        e = cudaEventRecord(g.la_ev[0], g.stream);
+        if (e != cudaSuccess) return e;
+    }
+    e = launch_chain_on<LOSS>(g, P[0]); // enqueued before the side stream's work: it takes its SMs first
+    if (e != cudaSuccess) return e;
+    if (n_slices > 1) {
+        e = cudaStreamWaitEvent(g.la_stream, g.la_ev[0], 0);
+        for (int s = 1; s < n_slices && e == cudaSuccess; ++s) {
+            e = launch_prepare_on<LOSS>(g, P[s], g.la_stream);
+            if (e == cudaSuccess) e = cudaEventRecord(g.la_ev[s], g.la_stream);
+        }
+        for (int s = 1; s < n_slices && e == cudaSuccess; ++s) {
+            e = cudaStreamWaitEvent(g.stream, g.la_ev[s], 0);
+            if (e == cudaSuccess) e = launch_chain_on<LOSS>(g, P[s]);
+        }
+    }
+    return e;
 }
 
 } // namespace
 
 int lookahead_max_dense_dim() { return kCapL; }
 
+// A round of many blocks is cut into this many slices at most (see launch_slices).
+constexpr int kMaxSlices = 3;
+int lookahead_max_slices() { return kMaxSlices; }
+
 // Bytes of the record buffer and of the block directory that a problem of this shape needs (every block's record at
-// its largest: a head, and 16 bytes per non-zero for the row-wise and the transposed copy).
+// its largest: a head, and 16 bytes per non-zero for the row-wise and the transposed copy; every slice may end in a
+// ragged block per partition).
 void lookahead_workspace(int64_t n_coord, int64_t nnz, int32_t K, bool dense, int64_t dim, size_t *rec_bytes, size_t *dir_bytes)
 {
-    const size_t max_blocks = (size_t)(n_coord / kLB + K + 1);
+    const size_t max_blocks = (size_t)(n_coord / kLB + (int64_t)kMaxSlices * (K + 1));
     *dir_bytes = max_blocks * sizeof(BlkDir);
     *rec_bytes = max_blocks * (sizeof(BlkHead) + 32) + (dense ? (size_t)n_coord * (size_t)dim * 4 : (size_t)nnz * 16) + 256;
 }
 
 cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
 {
-    LookParams P{};
-    P.S = S;
-    P.rec = static_cast<unsigned char *>(g.la_rec);
-    P.dir = static_cast<BlkDir *>(g.la_dir);
-    P.cursor = g.la_cursor;
-    P.rec_cap = g.la_rec_bytes;
-    P.blk_base = g.la_blk_base;
-    P.K = g.K;
-    P.n_blocks = 0;
-    for (int32_t k = 0; k < g.K; ++k) {
+    const int32_t K = g.K;
+    std::vector<int64_t> steps((size_t)K), nb((size_t)K);
+    int64_t total = 0, min_nb = (int64_t)1 << 62;
+    for (int32_t k = 0; k < K; ++k) {
         const int64_t nk = g.h_part_off[k + 1] - g.h_part_off[k];
-        const int64_t steps = g.round_steps ? g.round_steps[k] : (S.H == 0 ? nk : S.H);
-        P.n_blocks += (steps + kLB - 1) / kLB;
+        steps[(size_t)k] = g.round_steps ? g.round_steps[k] : (S.H == 0 ? nk : S.H);
+        nb[(size_t)k] = (steps[(size_t)k] + kLB - 1) / kLB;
+        total += nb[(size_t)k];
+        if (nb[(size_t)k] > 0 && nb[(size_t)k] < min_nb) min_nb = nb[(size_t)k];
     }
-    k_block_bases<<<1, 32, 0, g.stream>>>(S, g.K, g.la_blk_base);
-    if (P.n_blocks <= 0 || P.n_blocks > 0x7fffffff) return cudaErrorInvalidConfiguration;
+    if (total <= 0 || total > 0x7fffffff) return cudaErrorInvalidConfiguration;
+    // Long walks are cut into slices so that all but the first slice's prepare work runs beside the chain kernels
+    // (which occupy K SMs only; with more than half of the SMs taken by chains the prepare kernels would hold the
+    // chains up instead: such rounds stay in one piece). CHICLE_LA_SLICES=1 keeps every round in one piece (to time the prepare kernel alone),
+    // CHICLE_LA_SLICES=3 cuts short walks too (to test the slicing on small problems).
+    const bool can_slice = g.la_stream && g.la_slice && min_nb >= 8; // every partition has blocks in every slice
+    int n_slices = (can_slice && total >= 4096 && min_nb >= 64 && 2 * K <= g.sm_count) ? kMaxSlices : 1;
+    const char *env = getenv("CHICLE_LA_SLICES");
+    if (env && env[0] == '1' && env[1] == 0) n_slices = 1;
+    if (env && env[0] == '3' && env[1] == 0 && can_slice) n_slices = kMaxSlices;
+
+    LookParams P[kMaxSlices];
+    for (int s = 0; s < kMaxSlices; ++s) {
+        P[s] = LookParams{};
+        P[s].S = S;
+        P[s].rec = static_cast<unsigned char *>(g.la_rec);
+        P[s].cursor = g.la_cursor;
+        P[s].rec_cap = g.la_rec_bytes;
+        P[s].K = K;
+    }
+    cudaError_t e = cudaMemsetAsync(g.la_cursor, 0, sizeof(unsigned long long), g.stream);
+    if (e != cudaSuccess) return e;
+    if (n_slices == 1) {
+        P[0].dir = static_cast<BlkDir *>(g.la_dir);
+        P[0].blk_base = g.la_blk_base;
+        P[0].n_blocks = total;
+        k_block_bases<<<1, 32, 0, g.stream>>>(P[0].S, K, g.la_blk_base);
+    } else {
+        // slice s of partition k: blocks cut[s] .. cut[s + 1] of its walk, cut = 0, 1/8, 1/2, all of its blocks
+        std::vector<int64_t> h((size_t)kMaxSlices * 2 * (size_t)K);
+        int64_t blocks[kMaxSlices] = {0, 0, 0};
+        for (int32_t k = 0; k < K; ++k) {
+            const int64_t cut[kMaxSlices + 1] = {0, nb[(size_t)k] / 8, nb[(size_t)k] / 2, nb[(size_t)k]};
+            for (int s = 0; s < kMaxSlices; ++s) {
+                const int64_t first = cut[s] * kLB;
+                const int64_t last = s + 1 == kMaxSlices ? steps[(size_t)k] : cut[s + 1] * kLB;
+                h[((size_t)s * 2) * (size_t)K + (size_t)k] = last - first;
+                h[((size_t)s * 2 + 1) * (size_t)K + (size_t)k] = first;
+                blocks[s] += (last - first + kLB - 1) / kLB;
+            }
+        }
+        // a pageable source: the runtime has taken its copy of these words when the call returns
+        e = cudaMemcpyAsync(g.la_slice, h.data(), h.size() * sizeof(int64_t), cudaMemcpyHostToDevice, g.stream);
+        if (e != cudaSuccess) return e;
+        int64_t dir_off = 0;
+        for (int s = 0; s < kMaxSlices; ++s) {
+            P[s].S.H = 0;
+            P[s].S.steps_k = g.la_slice + ((size_t)s * 2) * (size_t)K;
+            P[s].S.first_k = g.la_slice + ((size_t)s * 2 + 1) * (size_t)K;
+            P[s].dir = static_cast<BlkDir *>(g.la_dir) + dir_off;
+            int64_t *bases = g.la_blk_base + (size_t)s * ((size_t)K + 1);
+            P[s].blk_base = bases;
+            P[s].n_blocks = blocks[s];
+            dir_off += blocks[s];
+            k_block_bases<<<1, 32, 0, g.stream>>>(P[s].S, K, bases);
+        }
+    }
     switch (g.loss) {
-    case CHICLE_LOSS_HINGE_DUAL: return launch_loss<CHICLE_LOSS_HINGE_DUAL>(g, P);
-    case CHICLE_LOSS_LOGISTIC_DUAL: return launch_loss<CHICLE_LOSS_LOGISTIC_DUAL>(g, P);
-    default: return launch_loss<CHICLE_LOSS_RIDGE_PRIMAL>(g, P);
+    case CHICLE_LOSS_HINGE_DUAL: return launch_slices<CHICLE_LOSS_HINGE_DUAL>(g, P, n_slices);
+    case CHICLE_LOSS_LOGISTIC_DUAL: return launch_slices<CHICLE_LOSS_LOGISTIC_DUAL>(g, P, n_slices);
+    default: return launch_slices<CHICLE_LOSS_RIDGE_PRIMAL>(g, P, n_slices);
     }
 }
 

@@ -110,6 +110,8 @@ struct SolverParams {
     uint32_t *status;
     int64_t n_coord, dim, H;
     const int64_t *steps_k; // K step budgets of this round, one per partition (each at most its size), or nullptr: H rules
+    const int64_t *first_k; // look-ahead solver only: where in its visiting order each partition starts in this launch
+                            // (a round cut into slices), or nullptr: at the start
     float lam_n, inv_n, lambda, sigma;
     int cap, nslot, multi_epoch;
 };

@@ -149,6 +149,26 @@ def test_rounds_of_several_local_epochs(monkeypatch):
     run_parity(tiny_csr(400, 40, seed=8, K=3), H=700, sizes=[50, 300, 50])
 
 
+def test_rounds_cut_into_slices(monkeypatch):
+    # long walks are cut into three slices whose prepare kernels run beside the chain kernels; forced here on walks the
+    # oracle finishes in seconds (at least 8 blocks per partition): all losses, unequal partitions, step budgets with an
+    # idle partition, several local epochs, and a walk too short to cut
+    monkeypatch.setenv("CHICLE_LA_SLICES", "3")
+    w = datagen.make("hinge_csr", 100)
+    run_parity(w, rounds=4)
+    n_k = w.n_coord // w.phases[0].K
+    run_parity(w, rounds=2, H=2 * n_k + 300)
+    K = w.phases[0].K
+    sizes = [n_k + (256 if k % 2 else -256) for k in range(K)]
+    run_parity(w, rounds=3, sizes=sizes, steps=lambda r: [0 if (k + r) % 7 == 0 else s - 20 * k for k, s in enumerate(sizes)])
+    run_parity(datagen.make("hinge_dense", 4), rounds=3)
+    run_parity(datagen.make("logistic_dense", 100), rounds=2)
+    run_parity(datagen.make("hinge_hashed", 1000), rounds=2)
+    w = datagen.make("ridge_csc", 100)
+    run_parity(w, rounds=2)
+    run_parity(tiny_csr(100, 30, seed=5, K=4))
+
+
 def test_ridge_small_with_long_and_empty_columns():
     rng = np.random.default_rng(11)
     n, d = 300, 500
