@@ -349,8 +349,11 @@ static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed,
     int64_t *h_off = h->h_part_off;
     const bool regrow = K != h->K || !h->U;
     if (regrow) {
-        // synchronise before releasing buffers that queued kernels may still use
+        // synchronise before releasing buffers that queued kernels may still use (the side stream's kernels are
+        // ordered before the end of the caller's stream in every round that completed; after a failed launch they
+        // may not be)
         e = cudaStreamSynchronize(h->stream);
+        if (e == cudaSuccess && h->la_stream) e = cudaStreamSynchronize(h->la_stream);
         if (e != cudaSuccess) return fail_cuda(h, e, "stream synchronise");
         float *newU = nullptr;
         int64_t *new_off = nullptr;
