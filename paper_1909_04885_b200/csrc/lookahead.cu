@@ -1123,11 +1123,15 @@ cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
         P[0].n_blocks = total;
         k_block_bases<<<1, 32, 0, g.stream>>>(P[0].S, K, g.la_blk_base);
     } else {
-        // slice s of partition k: blocks cut[s] .. cut[s + 1] of its walk, cut = 0, 1/8, 1/2, all of its blocks
+        // slice s of partition k: blocks cut[s] .. cut[s + 1] of its walk, cut = 0, 3/16, 13/16, all of its blocks.
+        // Measured: while prepare CTAs are pending, a finished chain launch's SMs are taken by them (four small CTAs
+        // per SM) and the next chain launch's CTAs, which need a whole SM each, get none until the prepare kernels
+        // run out of CTAs. So the first chain launch should last about as long as all the later slices' prepare
+        // work: 3/16 of the walk at 1.3 ms of prepare work against 6.3 ms of chain work per round.
         std::vector<int64_t> h((size_t)kMaxSlices * 2 * (size_t)K);
         int64_t blocks[kMaxSlices] = {0, 0, 0};
         for (int32_t k = 0; k < K; ++k) {
-            const int64_t cut[kMaxSlices + 1] = {0, nb[(size_t)k] / 8, nb[(size_t)k] / 2, nb[(size_t)k]};
+            const int64_t cut[kMaxSlices + 1] = {0, nb[(size_t)k] * 3 / 16, nb[(size_t)k] * 13 / 16, nb[(size_t)k]};
             for (int s = 0; s < kMaxSlices; ++s) {
                 const int64_t first = cut[s] * kLB;
                 const int64_t last = s + 1 == kMaxSlices ? steps[(size_t)k] : cut[s + 1] * kLB;
