@@ -244,14 +244,11 @@ template <int NZ, int HT, int THREADS> struct PreShared {
     unsigned long long offset;
 };
 
+// One block's record (all threads of the CTA; every return below is taken by all of them).
 template <int LOSS, int NZ, int HT, int THREADS>
-__global__ void __launch_bounds__(THREADS, 1024 / THREADS) k_lookahead_prepare(const LookParams P)
+__device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t bid, PreShared<NZ, HT, THREADS> &sh)
 {
-    extern __shared__ __align__(16) unsigned char smem_pre[];
-    using Shared = PreShared<NZ, HT, THREADS>;
-    Shared &sh = *reinterpret_cast<Shared *>(smem_pre);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t bid = blockIdx.x;
     int k;
     int64_t b;
     block_to_part(P, bid, k, b);
@@ -482,6 +479,21 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) k_lookahead_prepare(c
     PRE_T(7);
 }
 
+// A CTA takes blocks blockIdx.x, blockIdx.x + gridDim.x, ...: one each when the grid has a CTA per block; a launch
+// beside the chain kernels gets a grid that fits the SMs they leave, so that it never has CTAs waiting for an SM (which
+// would take the SMs of a finished chain launch before the next chain launch's CTAs, which need a whole SM each).
+template <int LOSS, int NZ, int HT, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) k_lookahead_prepare(const LookParams P)
+{
+    extern __shared__ __align__(16) unsigned char smem_pre[];
+    using Shared = PreShared<NZ, HT, THREADS>;
+    Shared &sh = *reinterpret_cast<Shared *>(smem_pre);
+    for (int64_t bid = blockIdx.x; bid < P.n_blocks; bid += gridDim.x) {
+        prepare_block<LOSS, NZ, HT, THREADS>(P, bid, sh);
+        __syncthreads(); // the shared arrays are reused by the next block
+    }
+}
+
 // Short dense rows: every row has every id, so the lists are implicit: headers, Gram triangle and the rows.
 struct PreDenseShared {
     float row[kLB][kCapL + 1];
@@ -490,11 +502,9 @@ struct PreDenseShared {
     uint32_t bytes;
 };
 
-template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_prepare_dense(const LookParams P)
+template <int LOSS> __device__ __forceinline__ void prepare_block_dense(const LookParams &P, const int64_t bid, PreDenseShared &sh)
 {
-    __shared__ PreDenseShared sh;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t bid = blockIdx.x;
     int k;
     int64_t b;
     block_to_part(P, bid, k, b);
@@ -555,6 +565,16 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) q0 += __shfl_xor_sync(0xffffffffu, q0, o);
         if (lane == 0 && j < cnt) out.hdr[j].q0 = q0;
+    }
+}
+
+// (blocks blockIdx.x, blockIdx.x + gridDim.x, ...: see k_lookahead_prepare)
+template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_prepare_dense(const LookParams P)
+{
+    __shared__ PreDenseShared sh;
+    for (int64_t bid = blockIdx.x; bid < P.n_blocks; bid += gridDim.x) {
+        prepare_block_dense<LOSS>(P, bid, sh);
+        __syncthreads();
     }
 }
 
@@ -1006,15 +1026,24 @@ template <int LOSS, int NZ, int HT, int THREADS> cudaError_t launch_prepare(Glm 
 template <int LOSS> cudaError_t launch_prepare_on(Glm &g, const LookParams &P, cudaStream_t stream)
 {
     const unsigned nb = (unsigned)P.n_blocks;
+    // beside the chain kernels: no more CTAs than fit the SMs the chains leave (see k_lookahead_prepare)
+    const unsigned free_sms = (unsigned)(g.sm_count > g.K ? g.sm_count - g.K : 1);
     if (g.fmt == CHICLE_FMT_DENSE_ROWMAJOR) {
-        k_lookahead_prepare_dense<LOSS><<<nb, kPreThreads, 0, stream>>>(P);
+        const unsigned per_sm = 2048 / kPreThreads;
+        const unsigned grid = stream == g.stream || nb < free_sms * per_sm ? nb : free_sms * per_sm;
+        k_lookahead_prepare_dense<LOSS><<<grid, kPreThreads, 0, stream>>>(P);
         return cudaGetLastError();
     }
     // blocks of up to 2 048 non-zeros (32 coordinates of 50 on average, with room): the small variant, four CTAs per SM
     const double avg_block = 32.0 * (double)g.nnz / (double)g.n_coord;
     cudaError_t e;
-    if (avg_block * 1.25 <= 2048.0) e = launch_prepare<LOSS, 2048, 2048, 256>(g, P, nb, stream);
-    else e = launch_prepare<LOSS, kMaxNz, kHT, kPreThreadsS>(g, P, nb, stream);
+    if (avg_block * 1.25 <= 2048.0) {
+        const unsigned grid = stream == g.stream || nb < free_sms * 4 ? nb : free_sms * 4;
+        e = launch_prepare<LOSS, 2048, 2048, 256>(g, P, grid, stream);
+    } else {
+        const unsigned grid = stream == g.stream || nb < free_sms * 2 ? nb : free_sms * 2;
+        e = launch_prepare<LOSS, kMaxNz, kHT, kPreThreadsS>(g, P, grid, stream);
+    }
 #ifdef CHICLE_LA_TIMING
     if (e == cudaSuccess) {
         unsigned long long t[8] = {0};
@@ -1123,15 +1152,27 @@ cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
         P[0].n_blocks = total;
         k_block_bases<<<1, 32, 0, g.stream>>>(P[0].S, K, g.la_blk_base);
     } else {
-        // slice s of partition k: blocks cut[s] .. cut[s + 1] of its walk, cut = 0, 3/16, 13/16, all of its blocks.
-        // Measured: while prepare CTAs are pending, a finished chain launch's SMs are taken by them (four small CTAs
-        // per SM) and the next chain launch's CTAs, which need a whole SM each, get none until the prepare kernels
-        // run out of CTAs. So the first chain launch should last about as long as all the later slices' prepare
-        // work: 3/16 of the walk at 1.3 ms of prepare work against 6.3 ms of chain work per round.
+        // Slice s of partition k: blocks cut[s] .. cut[s + 1] of its walk. The prepare kernel of slice s + 1 should
+        // be done when the chain launch of slice s is, so the slices grow by a factor a = 0.8 / rho, where rho is the
+        // prepare time of a piece of the walk on the SMs the chains leave over its chain time: about
+        // c K / (SMs - K) with c = SM-time of the prepare kernel per step over the chain's time per step, 1.2 to
+        // 1.9 measured on the sparse configurations (2 assumed), 0.18 on short dense rows (0.25 assumed). The first
+        // slice's prepare kernel is the part that stays exposed: 1 / (1 + a + a^2) of the walk.
+        const double c_ratio = g.fmt == CHICLE_FMT_DENSE_ROWMAJOR ? 0.25 : 2.0;
+        const double rho = c_ratio * (double)K / (double)(g.sm_count > K ? g.sm_count - K : 1);
+        const double a = 0.8 / rho;
+        double f1 = 1.0 / (1.0 + a + a * a);
+        f1 = f1 < 1.0 / 64 ? 1.0 / 64 : (f1 > 0.5 ? 0.5 : f1);
+        const double f2 = a * f1;
         std::vector<int64_t> h((size_t)kMaxSlices * 2 * (size_t)K);
         int64_t blocks[kMaxSlices] = {0, 0, 0};
         for (int32_t k = 0; k < K; ++k) {
-            const int64_t cut[kMaxSlices + 1] = {0, nb[(size_t)k] * 3 / 16, nb[(size_t)k] * 13 / 16, nb[(size_t)k]};
+            const int64_t nbk = nb[(size_t)k]; // 0, or at least 8
+            int64_t c1 = (int64_t)((double)nbk * f1), c2 = (int64_t)((double)nbk * (f1 + f2));
+            c1 = c1 < 1 ? 1 : c1;
+            c2 = c2 < c1 + 1 ? c1 + 1 : c2;
+            c2 = c2 > nbk - 1 ? nbk - 1 : c2;
+            const int64_t cut[kMaxSlices + 1] = {0, nbk ? c1 : 0, nbk ? c2 : 0, nbk};
             for (int s = 0; s < kMaxSlices; ++s) {
                 const int64_t first = cut[s] * kLB;
                 const int64_t last = s + 1 == kMaxSlices ? steps[(size_t)k] : cut[s + 1] * kLB;

@@ -161,6 +161,8 @@ def test_rounds_cut_into_slices(monkeypatch):
     K = w.phases[0].K
     sizes = [n_k + (256 if k % 2 else -256) for k in range(K)]
     run_parity(w, rounds=3, sizes=sizes, steps=lambda r: [0 if (k + r) % 7 == 0 else s - 20 * k for k, s in enumerate(sizes)])
+    # a slice of more blocks than the prepare kernel's grid beside the chains has CTAs: its CTAs take several blocks each
+    run_parity(datagen.make("hinge_csr", 10), rounds=2, check_perm=False)
     run_parity(datagen.make("hinge_dense", 4), rounds=3)
     run_parity(datagen.make("logistic_dense", 100), rounds=2)
     run_parity(datagen.make("hinge_hashed", 1000), rounds=2)
