@@ -1,7 +1,7 @@
 /*
  * chicle.h -- C ABI of libchicle: one CoCoA round for generalised linear models on one NVIDIA B200.
  *
- * A round (paper Sec. 2.1, Eq. 1 and Eq. 2; Sec. 2.2 "CoCoA"; Sec. 5.1 "CoCoA"): K uni-task partitions of the
+ * A round (paper Sec. 2.2, Eq. 1, Eq. 2 and "CoCoA"; Sec. 5.1 "CoCoA"): K uni-task partitions of the
  * coordinates each run a sequential stochastic coordinate-descent solver against a private copy of the shared
  * vector v, the K updates are added into v, and the duality gap (the paper's convergence metric, Sec. 4.1 and
  * Sec. 5) can be evaluated. Every step runs in CUDA kernels of this library; there is no host fallback.
@@ -103,8 +103,8 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
                                   int device, void *cuda_stream, const chicle_allocator_t *alloc,
                                   chicle_glm_t **out);
 
-/* Random equal split of the coordinates into K disjoint covering partitions (Sec. 2.1: disjoint partitions D_k;
- * Sec. 3: the data parallelism can change between iterations; Sec. 6: data is assigned to tasks at random).
+/* Random equal split of the coordinates into K disjoint covering partitions (Sec. 2.2: disjoint partitions D_k;
+ * Sec. 3: the data parallelism can change between iterations; Appendix, baseline comparisons: data is assigned to tasks at random).
  * Integer rule: ids are ordered by mix64(mix64(seed) ^ id) (mix64 = one SplitMix64 output for that state) and
  * cut into K consecutive blocks, the first n mod K one longer. 1 <= K <= number of coordinates. Legal only
  * between rounds; keeps alpha, v and the round counter; (re)allocates the per-partition workspaces. */
@@ -120,7 +120,7 @@ chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed);
 chicle_status_t chicle_partition_sizes(chicle_glm_t *h, int32_t K, uint64_t seed, const int64_t *host_sizes);
 
 /* ---- mobile data chunks (Sec. 3 core concepts: the samples live in many small fixed-size chunks that the scheduler
- * moves between immobile tasks; Sec. 4.3: a chunk holds samples and their per-sample state, their number varies with
+ * moves between immobile tasks; Sec. 4.4: a chunk holds samples and their per-sample state, their number varies with
  * their size). The five functions below are host-side integer logic: all pointers are HOST arrays, no GPU is touched,
  * no handle is needed. A placement is `chunk_off` (n_chunks + 1 ascending coordinate offsets, chunk c = coordinates
  * chunk_off[c] .. chunk_off[c+1]-1 in id order) and `chunk_task` (n_chunks task numbers). The paper fixes none of the
@@ -133,7 +133,7 @@ chicle_status_t chicle_partition_sizes(chicle_glm_t *h, int32_t K, uint64_t seed
 int64_t chicle_chunks_cut(int64_t n_coord, const int64_t *host_indptr, int64_t dense_dim, int64_t chunk_bytes,
                           int64_t *host_chunk_off);
 
-/* First placement (Sec. 6: data is assigned to tasks at random): the chunks, ordered by (mix64(mix64(seed) ^ chunk),
+/* First placement (Appendix, baseline comparisons: data is assigned to tasks at random): the chunks, ordered by (mix64(mix64(seed) ^ chunk),
  * chunk), are dealt in K consecutive runs, the first n_chunks mod K tasks getting one more. 1 <= K <= n_chunks. */
 chicle_status_t chicle_chunks_assign(int64_t n_chunks, int32_t K, uint64_t seed, int32_t *host_chunk_task);
 
@@ -161,14 +161,14 @@ int chicle_chunks_rebalance_step(int64_t n_chunks, const int64_t *host_chunk_off
 
 /* The partition a placement induces: coordinate i belongs to the task of its chunk; members in ascending id order
  * inside a partition (the owner map and the member lists are built on the device). Otherwise as chicle_partition:
- * legal between rounds, keeps alpha, v and the round counter (the state moves with the samples, Sec. 4.3); `seed` keys
+ * legal between rounds, keeps alpha, v and the round counter (the state moves with the samples, Sec. 4.4); `seed` keys
  * the visiting orders of the rounds that follow. K <= n_chunks <= coordinates, offsets from 0 to the number of
  * coordinates and strictly increasing, tasks in [0, K), every task holding a chunk: else CHICLE_ERR_INVALID_ARG and
  * the handle is unchanged. The host arrays are read during the call. */
 chicle_status_t chicle_partition_chunks(chicle_glm_t *h, int32_t K, uint64_t seed, int64_t n_chunks,
                                         const int64_t *host_chunk_off, const int32_t *host_chunk_task);
 
-/* One CoCoA round (Sec. 2.1 Eq. 1, Eq. 2 and worker structure with L = 1; Sec. 5.1: SCD local solver, sigma =
+/* One CoCoA round (Sec. 2.2 Eq. 1, Eq. 2 and worker structure with L = 1; Sec. 5.1: SCD local solver, sigma =
  * number of tasks). Each partition draws this round's seeded visiting order (members ordered by
  * mix64(mix64(seed ^ 0xD1B54A32D192ED03) ^ mix64(round * 2^32 + epoch) ^ id)), walks it strictly in order for H
  * coordinate steps (H = 0: one local epoch, i.e. as many steps as the partition has coordinates) against

@@ -163,7 +163,7 @@ class CocoaOracle:
         self.K, self.seed = int(K), int(seed)
 
     def partition_chunks(self, K: int, seed: int, chunk_off, chunk_task):
-        """The partition that a placement of data chunks on K tasks induces (Sec. 3, Sec. 4.3); ``seed`` keys the
+        """The partition that a placement of data chunks on K tasks induces (Sec. 3, Sec. 4.4); ``seed`` keys the
         visiting orders of the rounds that follow."""
         from . import chunks
         self.owner, self.part_off, self.members = chunks.partition_from_chunks(self.n_coord, K, chunk_off, chunk_task)

@@ -1,7 +1,7 @@
 """Test infrastructure (CPU oracle): mobile data chunks and the elastic policies that move them between tasks.
 
 The paper keeps the training data in many small fixed-size chunks that carry the samples together with their
-per-sample state (Sec. 3 core concepts; Sec. 4.3 in-memory chunk format: the number of samples in a chunk varies with
+per-sample state (Sec. 3 core concepts; Sec. 4.4 in-memory chunk format: the number of samples in a chunk varies with
 their size). Tasks never move; the scheduler moves chunks: when tasks are freed their chunks go to the remaining
 tasks in round-robin fashion (Sec. 4.5 elastic scaling policy), when tasks are added each old task hands randomly
 picked chunks to the new ones (Sec. 5.3: this is why scaling out reshuffles the samples), and the rebalancing policy
@@ -19,7 +19,7 @@ SCALE_OUT_STREAM = 0xA0761D6478BD642F
 
 
 def cut(n_coord, chunk_bytes, indptr=None, dense_dim=0):
-    """Chunk boundaries (Sec. 4.3). Coordinates are stored in id order. Coordinate i occupies
+    """Chunk boundaries (Sec. 4.4). Coordinates are stored in id order. Coordinate i occupies
     NNZ_BYTES * nnz_i + STATE_BYTES bytes (sparse) or 4 * dense_dim + STATE_BYTES (dense). A chunk is closed in front of
     the coordinate that would take it above chunk_bytes; a chunk holds at least one coordinate. Returns off[C + 1]."""
     off = [0]
@@ -35,7 +35,7 @@ def cut(n_coord, chunk_bytes, indptr=None, dense_dim=0):
 
 
 def assign(C, K, seed):
-    """First placement (Sec. 6: data is assigned to tasks at random): the chunks, ordered by
+    """First placement (Appendix, baseline comparisons: data is assigned to tasks at random): the chunks, ordered by
     mix64(mix64(seed) ^ chunk), are dealt in consecutive runs, the first C mod K tasks getting one more."""
     if not 1 <= K <= C:
         raise ValueError("need 1 <= K <= number of chunks")

@@ -6,9 +6,9 @@
  * and called by the tests, the smoke check and the benchmark's CPU-baseline leg.
  *
  * What it follows (paper sections):
- *   - Sec. 2.1, Eq. 1 and Eq. 2: an iteration refines the shared model from K local updates that are
+ *   - Sec. 2.2, Eq. 1 and Eq. 2: an iteration refines the shared model from K local updates that are
  *     computed independently on K disjoint partitions and then combined.
- *   - Sec. 2.1 (worker structure, Fig. 2): each worker takes H sequential steps of L samples and updates
+ *   - Sec. 2.2 (worker structure, Fig. 2): each worker takes H sequential steps of L samples and updates
  *     its local model after every step, so later steps see earlier ones.
  *   - Sec. 2.2 "CoCoA": L = 1, the local optimiser is SCD over the partition, K is the data parallelism.
  *   - Sec. 5.1 "CoCoA": SVM trained with SCD, H = number of local samples, sigma = number of tasks.
@@ -25,8 +25,10 @@
  * Parity pins (tests/test_oracle_pins.py): mix64 against the published SplitMix64 outputs; partition and
  * permutation against their defining properties; hinge against a brute-force QP; ridge against the normal
  * equations; logistic against bisection and a Newton solve of the primal; K=1 against a separately written
- * SDCA loop; orthogonal rows against the closed form; Fenchel-Young non-negativity; v == X^T alpha;
- * dual ascent; repartition invariance. Parity with the paper's own (unreleased) implementation and its
+ * SDCA loop; orthogonal rows against the closed form; the sigma' factor of the local model by a K = 2,
+ * sigma' = 2 case worked by hand and by every step maximising its task's explicitly evaluated sigma'-subproblem
+ * along its coordinate; Fenchel-Young non-negativity; v == X^T alpha; dual ascent; weak duality across
+ * rounds; repartition invariance. Parity with the paper's own (unreleased) implementation and its
  * random streams: parity unpinned.
  */
 #include <math.h>
@@ -38,8 +40,6 @@
 #endif
 
 enum { ORC_HINGE = 0, ORC_LOGISTIC = 1, ORC_RIDGE = 2 };
-
-#define ORC_NEWTON_ITERS 5
 
 /* ---- integer part: mixer, partition, permutation -------------------------------------------------- */
 
@@ -72,8 +72,8 @@ static int orc_i32_cmp(const void *pa, const void *pb)
     return (a > b) - (a < b);
 }
 
-/* Random equal split of coordinates 0..n-1 into K disjoint covering partitions (Sec. 2.1: disjoint
- * partitions D_k; Sec. 5/6: random assignment of data to tasks). Sort ids by (mix64(mix64(seed) ^ id), id),
+/* Random equal split of coordinates 0..n-1 into K disjoint covering partitions (Sec. 2.2: disjoint
+ * partitions D_k; Appendix, baseline comparisons: random assignment of data to tasks). Sort ids by (mix64(mix64(seed) ^ id), id),
  * cut the sorted list into K consecutive blocks, the first n mod K blocks one longer; inside a partition
  * the members are listed in ascending id.  Returns 0, or -1 on bad arguments / out of memory. */
 static int orc_partition_cut(int64_t n, int32_t K, uint64_t seed, const int64_t *sizes, int32_t *owner, int64_t *part_off,
@@ -212,37 +212,31 @@ double orc_step_hinge(double a, double m, double q)
 }
 
 /* Logistic: maximise  -[a' log a' + (1-a') log(1-a')] - (a'-a) m - (q/2)(a'-a)^2  over a' in (0,1).
- * With a' = sigmoid(z) the stationarity condition is  z + q sigmoid(z) = c,  c = q a - m.  The recipe is
- * fixed so that the checker and the library take the same steps:
- *   1. If c > q/2 the root is positive: substitute z -> -z, c -> q - c (sigmoid(-z) = 1 - sigmoid(z)), so
- *      that from here on the root is <= 0, where F(z) = z + q sigmoid(z) - c is convex and increasing.
- *   2. Start: with kappa = log q + c, z0 = min(c, 0) if kappa <= 0 (linear part dominates), else
- *      z0 = min(c - (kappa - log(1 + kappa)), 0) (exponential part dominates; a rough Lambert-W value).
- *   3. ORC_NEWTON_ITERS Newton steps z <- min(z - F/F', 0), F' = 1 + q p (1 - p), p = sigmoid(z).
- *      On a convex increasing F Newton's iterates are to the right of the root after the first step and
- *      decrease monotonically to it; the cap at 0 keeps them on the convex branch.
- *   4. a' = sigmoid(z), or 1 - sigmoid(z) if step 1 substituted.
- * q = 0 (zero row) gives a' = sigmoid(-m) exactly. The residual F at the returned point is written to
- * *resid when resid != NULL. */
+ * With a' = sigmoid(z) the stationarity condition is  F(z) = z + q sigmoid(z) - c = 0,  c = q a - m.
+ * F is continuous and strictly increasing (F' = 1 + q p (1-p) >= 1), and since 0 <= sigmoid <= 1 the unique
+ * root lies in [c - q, c]. It is found the plain way: a bracket [lo, hi] with F(lo) <= 0 <= F(hi) that every
+ * evaluation narrows; the next point is Newton's when that falls strictly inside the bracket, else the
+ * midpoint; stop when |F| <= 1e-12 or the bracket has no interior point in fp64 (for |c| of 1e4 and more the
+ * spacing of doubles near the root is itself above 1e-12). q = 0 (zero row) gives a' = sigmoid(-m) exactly.
+ * The residual F at the returned point is written to *resid when resid != NULL. */
 double orc_step_logistic(double a, double m, double q, double *resid)
 {
-    double c = q * a - m;
-    const int flip = c > 0.5 * q;
-    if (flip) c = q - c;
-    double z;
-    const double kappa = (q > 0.0) ? log(q) + c : -INFINITY;
-    if (kappa <= 0.0) z = c < 0.0 ? c : 0.0;
-    else { z = c - (kappa - log1p(kappa)); if (z > 0.0) z = 0.0; }
-    for (int it = 0; it < ORC_NEWTON_ITERS; ++it) {
+    const double c = q * a - m;
+    double lo = c - q, hi = c;
+    double z = 0.5 * (lo + hi);
+    for (int it = 0; it < 400; ++it) {
         const double p = orc_sigmoid(z);
         const double F = z + q * p - c;
-        const double Fp = 1.0 + q * p * (1.0 - p);
-        z -= F / Fp;
-        if (z > 0.0) z = 0.0;
+        if (fabs(F) <= 1e-12) break;
+        if (F > 0.0) hi = z; else lo = z;
+        double zn = z - F / (1.0 + q * p * (1.0 - p));
+        if (!(zn > lo && zn < hi)) zn = 0.5 * (lo + hi);
+        if (!(zn > lo && zn < hi)) break;   /* lo and hi are neighbouring doubles */
+        z = zn;
     }
     const double p = orc_sigmoid(z);
     if (resid) *resid = z + q * p - c;
-    return flip ? 1.0 - p : p;
+    return p;
 }
 
 static double orc_xlogx(double x) { return x > 0.0 ? x * log(x) : 0.0; }

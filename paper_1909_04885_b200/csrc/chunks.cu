@@ -1,5 +1,5 @@
 // Mobile data chunks: where the chunk boundaries fall and which task holds which chunk. Host-side integer logic of the
-// scheduler (the paper's Sec. 3 core concepts, Sec. 4.3 chunk format, Sec. 4.5 elastic scaling and rebalancing
+// scheduler (the paper's Sec. 3 core concepts, Sec. 4.4 chunk format, Sec. 4.5 elastic scaling and rebalancing
 // policies, Sec. 5.3 on how scaling out reshuffles); the placement these functions produce is turned into a partition
 // on the device by chicle_partition_chunks. No GPU is touched here.
 #include <algorithm>

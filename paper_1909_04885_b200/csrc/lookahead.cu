@@ -1,5 +1,5 @@
 // Local SCD solver with block look-ahead: the same result as walking a partition's visiting order coordinate by
-// coordinate (paper Sec. 2.1 worker structure with L = 1; Sec. 5.1: SCD local solver), up to rounding order, with
+// coordinate (paper Sec. 2.2 worker structure with L = 1; Sec. 5.1: SCD local solver), up to rounding order, with
 // the work that does not depend on earlier steps taken off the sequential chain.
 //
 // The walk is cut into blocks of 32 consecutive steps. Inside a block, with w the local model at the block's start,

@@ -1,5 +1,5 @@
 // Local stochastic coordinate-descent solvers: one CTA per partition, walking the partition's visiting order
-// strictly in order (paper Sec. 2.1 worker structure with L = 1; Sec. 2.2 and Sec. 5.1: SCD local solver).
+// strictly in order (paper Sec. 2.2 worker structure with L = 1 and "CoCoA"; Sec. 5.1: SCD local solver).
 //
 // Roles inside a CTA
 //   warp 0        the chain: per step one dot product (lanes over the coordinate's entries, butterfly

@@ -1,5 +1,5 @@
 // Local SCD solver for sparse coordinates (CSR rows / CSC columns) and for short dense rows: one CTA per partition, the visiting order
-// walked strictly in order (paper Sec. 2.1 worker structure with L = 1; Sec. 5.1: SCD local solver), with the
+// walked strictly in order (paper Sec. 2.2 worker structure with L = 1; Sec. 5.1: SCD local solver), with the
 // part of the local model that the next steps can touch held in shared memory.
 //
 // Local model: w_local = v + sigma' * U_k, where U_k (the partition's accumulated update, zero at round start) has

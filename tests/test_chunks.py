@@ -1,4 +1,4 @@
-"""Mobile data chunks and the elastic policies (Sec. 3, Sec. 4.3, Sec. 4.5, Sec. 5.3): the oracle's rules against
+"""Mobile data chunks and the elastic policies (Sec. 3, Sec. 4.4, Sec. 4.5, Sec. 5.3): the oracle's rules against
 hand-worked cases and their defining properties, and the library's host functions against the oracle, bit for bit."""
 import numpy as np
 import pytest
