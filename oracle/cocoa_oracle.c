@@ -215,24 +215,35 @@ double orc_step_hinge(double a, double m, double q)
  * With a' = sigmoid(z) the stationarity condition is  F(z) = z + q sigmoid(z) - c = 0,  c = q a - m.
  * F is continuous and strictly increasing (F' = 1 + q p (1-p) >= 1), and since 0 <= sigmoid <= 1 the unique
  * root lies in [c - q, c]. It is found the plain way: a bracket [lo, hi] with F(lo) <= 0 <= F(hi) that every
- * evaluation narrows; the next point is Newton's when that falls strictly inside the bracket, else the
- * midpoint; stop when |F| <= 1e-12 or the bracket has no interior point in fp64 (for |c| of 1e4 and more the
+ * evaluation narrows; the next point is Newton's when that falls strictly inside the bracket and the steps are
+ * at least halving, else the midpoint (the textbook safeguarded Newton iteration); stop when |F| <= 1e-12 or the bracket has no interior point in fp64 (for |c| of 1e4 and more the
  * spacing of doubles near the root is itself above 1e-12). q = 0 (zero row) gives a' = sigmoid(-m) exactly.
  * The residual F at the returned point is written to *resid when resid != NULL. */
 double orc_step_logistic(double a, double m, double q, double *resid)
 {
     const double c = q * a - m;
-    double lo = c - q, hi = c;
+    double lo = c - q, hi = c;              /* F(lo) <= 0 <= F(hi) */
     double z = 0.5 * (lo + hi);
+    double step_before = hi - lo, step = step_before;
     for (int it = 0; it < 400; ++it) {
         const double p = orc_sigmoid(z);
         const double F = z + q * p - c;
         if (fabs(F) <= 1e-12) break;
         if (F > 0.0) hi = z; else lo = z;
-        double zn = z - F / (1.0 + q * p * (1.0 - p));
-        if (!(zn > lo && zn < hi)) zn = 0.5 * (lo + hi);
-        if (!(zn > lo && zn < hi)) break;   /* lo and hi are neighbouring doubles */
-        z = zn;
+        const double Fp = 1.0 + q * p * (1.0 - p);
+        const double zn = z - F / Fp;
+        /* Newton's point if it lies inside the bracket and the steps are at least halving, else the midpoint */
+        if (zn > lo && zn < hi && fabs(2.0 * F) <= fabs(step_before * Fp)) {
+            step_before = step;
+            step = F / Fp;
+            z = zn;
+        } else {
+            step_before = step;
+            step = 0.5 * (hi - lo);
+            const double mid = lo + step;
+            if (!(mid > lo && mid < hi)) break;   /* lo and hi are neighbouring doubles */
+            z = mid;
+        }
     }
     const double p = orc_sigmoid(z);
     if (resid) *resid = z + q * p - c;

@@ -496,6 +496,19 @@ def test_logistic_step_against_bisection():
             assert abs(resid) <= 1e-9
             assert 0.0 <= got <= 1.0
     assert abs(oracle.step_logistic(0.3, 1.7, 0.0)[0] - sig(-1.7)) < 1e-15      # zero row
+    # the regime of the workloads: a anywhere in (0, 1), margins of a few units, q over six decades (here Newton's
+    # iteration from the middle of the bracket alternates between the two flat ends of the sigmoid)
+    for _ in range(20000):
+        q, a, m = float(10 ** rng.uniform(-3, 3)), float(rng.random()), float(3 * rng.standard_normal())
+        lo, hi = q * a - m - q, q * a - m
+        for _ in range(200):
+            mid = 0.5 * (lo + hi)
+            if mid + m + q * (sig(mid) - a) > 0:
+                hi = mid
+            else:
+                lo = mid
+        got, resid = oracle.step_logistic(a, m, q)
+        assert abs(got - sig(0.5 * (lo + hi))) < 1e-12 and abs(resid) <= 1e-9
 
 
 def test_logistic_converges_to_primal_minimiser():
