@@ -100,8 +100,12 @@ void destroy_impl(chicle_glm *h)
         (void)cudaStreamSynchronize(h->la_stream);
         (void)cudaStreamDestroy(h->la_stream);
     }
-    for (auto &ev : h->la_ev)
-        if (ev) (void)cudaEventDestroy(ev);
+    for (int i = 0; i < lookahead_max_slices(); ++i) {
+        if (h->la_ev_prep && h->la_ev_prep[i]) (void)cudaEventDestroy(h->la_ev_prep[i]);
+        if (h->la_ev_done && h->la_ev_done[i]) (void)cudaEventDestroy(h->la_ev_done[i]);
+    }
+    delete[] h->la_ev_prep;
+    delete[] h->la_ev_done;
     while (!h->owned.empty()) dev_free(h, h->owned.back());
     if (h->h_status) (void)cudaFreeHost(h->h_status);
     if (h->h_gap) (void)cudaFreeHost(h->h_gap);
@@ -205,8 +209,14 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
         (void)cudaDeviceGetStreamPriorityRange(&least, &greatest);
         if ((e = cudaStreamCreateWithPriority(&h->la_stream, cudaStreamNonBlocking, least)) != cudaSuccess)
             return bail_cuda(e, "cudaStreamCreateWithPriority");
-        for (auto &ev : h->la_ev)
-            if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return bail_cuda(e, "cudaEventCreate");
+        const int ns = lookahead_max_slices();
+        h->la_ev_prep = new (std::nothrow) cudaEvent_t[(size_t)ns]();
+        h->la_ev_done = new (std::nothrow) cudaEvent_t[(size_t)ns]();
+        if (!h->la_ev_prep || !h->la_ev_done) return bail(CHICLE_ERR_OOM, "host allocation failed");
+        for (int i = 0; i < ns; ++i)
+            if ((e = cudaEventCreateWithFlags(&h->la_ev_prep[i], cudaEventDisableTiming)) != cudaSuccess ||
+                (e = cudaEventCreateWithFlags(&h->la_ev_done[i], cudaEventDisableTiming)) != cudaSuccess)
+                return bail_cuda(e, "cudaEventCreate");
     }
 
     cudaStream_t s = h->stream;
@@ -374,19 +384,18 @@ static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed,
         U = newU; part_off = new_off; h_off = new_hoff;
         // the look-ahead solver's per-round records (their number depends on K); without them the blocked solver runs
         dev_free(h, h->la_rec); dev_free(h, h->la_dir); dev_free(h, h->la_cursor); dev_free(h, h->la_blk_base); dev_free(h, h->la_slice);
-        h->la_rec = nullptr; h->la_dir = nullptr; h->la_cursor = nullptr; h->la_blk_base = nullptr; h->la_slice = nullptr; h->la_rec_bytes = 0;
+        h->la_rec = nullptr; h->la_dir = nullptr; h->la_cursor = nullptr; h->la_blk_base = nullptr; h->la_slice = nullptr;
         const bool dense_fmt = h->fmt == CHICLE_FMT_DENSE_ROWMAJOR;
-        if (!dense_fmt || h->dim <= lookahead_max_dense_dim()) {
-            size_t rec_bytes = 0, dir_bytes = 0;
-            lookahead_workspace(n, h->nnz, K, dense_fmt, h->dim, &rec_bytes, &dir_bytes);
+        if (dense_fmt ? h->dim <= lookahead_max_dense_dim() : h->dim <= lookahead_max_dim()) {
+            lookahead_plan(*h, K);
             unsigned char *rec = nullptr, *dir = nullptr;
-            if (alloc_into(h, rec, rec_bytes) && alloc_into(h, dir, dir_bytes) && alloc_into(h, h->la_cursor, 32) &&
+            if (alloc_into(h, rec, (size_t)h->la_regions * h->la_region_bytes) && alloc_into(h, dir, h->la_dir_bytes) &&
+                alloc_into(h, h->la_cursor, 64) &&
                 alloc_into(h, h->la_blk_base, (size_t)lookahead_max_slices() * ((size_t)K + 1)) &&
                 alloc_into(h, h->la_slice, (size_t)lookahead_max_slices() * 2 * (size_t)K)) {
                 h->la_rec = rec;
                 h->la_dir = dir;
-                h->la_rec_bytes = rec_bytes;
-                (void)cudaMemsetAsync(h->la_cursor, 0, 32 * sizeof(unsigned long long), h->stream);
+                (void)cudaMemsetAsync(h->la_cursor, 0, 64 * sizeof(unsigned long long), h->stream);
             } else {
                 dev_free(h, rec); dev_free(h, dir); dev_free(h, h->la_cursor); dev_free(h, h->la_blk_base); dev_free(h, h->la_slice);
                 h->la_cursor = nullptr; h->la_blk_base = nullptr; h->la_slice = nullptr;

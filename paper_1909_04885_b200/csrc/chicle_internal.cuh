@@ -98,16 +98,23 @@ struct Glm {
     float *U = nullptr;         // K * dim: per-partition accumulated update, zero between rounds
     int64_t U_rows = 0;
 
-    // look-ahead solver: the per-block records that its prepare kernel writes every round, and where each one is
-    // (nullptr when they could not be allocated: the blocked solver runs instead)
+    // look-ahead solver: the per-block records that its prepare kernel writes every round (nullptr when they could
+    // not be allocated: the blocked solver runs instead). The buffer is a ring of regions, one slice of a round each.
     void *la_rec = nullptr;
-    void *la_dir = nullptr;
-    unsigned long long *la_cursor = nullptr;
-    size_t la_rec_bytes = 0;
-    int64_t *la_blk_base = nullptr; // per slice K+1: first block of each partition in the slice's numbering of the blocks
-    int64_t *la_slice = nullptr;    // per slice 2K: every partition's step count and first step in that slice
+    void *la_dir = nullptr;          // per region: cluster-size entries per block
+    unsigned long long *la_cursor = nullptr; // [r]: bytes of region r's pool handed out; [8..]: timing scratch
+    size_t la_region_bytes = 0, la_pool_off = 0, la_dir_bytes = 0;
+    int64_t la_region_blocks = 0;    // blocks a region has records for
+    int la_regions = 0;
+    int la_logC = 0;                 // log2 of the CTAs per partition (thread-block cluster)
+    int32_t la_nzcap = 0, la_hotc = 0; // non-zeros per worker record; entry ids per CTA kept in shared memory
+    size_t la_smem = 0;              // dynamic shared memory of the chain kernel
+    int la_last_slices = 0;          // slices of the last round
+    int64_t *la_blk_base = nullptr;  // per slice K+1: first block of each partition in the slice's numbering of the blocks
+    int64_t *la_slice = nullptr;     // per slice 2K: every partition's step count and first step in that slice
     cudaStream_t la_stream = nullptr; // side stream (lowest priority) for the later slices' prepare kernels
-    cudaEvent_t la_ev[3] = {nullptr, nullptr, nullptr}; // slice s is prepared
+    cudaEvent_t *la_ev_prep = nullptr; // per slice: its records are written
+    cudaEvent_t *la_ev_done = nullptr; // per slice: its chain launch is done (its region is free)
     bool time_prepare = false; // record ev[4] between the prepare and the chain kernel (round statistics asked for)
 
     SortWorkspace sortws;
@@ -140,9 +147,10 @@ cudaError_t launch_frequency_remap(Glm &g, uint32_t *counts, uint64_t *keys[2], 
                                    uint32_t *scan_sums, int64_t hot_ids, int32_t long_len, unsigned long long *mass);
 cudaError_t launch_gather_f32(Glm &g, const float *src, const int32_t *map, int64_t n, float *dst); // dst[i] = src[map[i]]
 cudaError_t launch_lookahead_solver(Glm &g, const struct SolverParams &P);
-void lookahead_workspace(int64_t n_coord, int64_t nnz, int32_t K, bool dense, int64_t dim, size_t *rec_bytes, size_t *dir_bytes);
+void lookahead_plan(Glm &g, int32_t K); // fills the la_* sizes for a partition into K
 int lookahead_max_dense_dim();
 int lookahead_max_slices();
+int64_t lookahead_max_dim();
 int blocked_solver_hot_ids();
 int blocked_solver_short_cap();
 

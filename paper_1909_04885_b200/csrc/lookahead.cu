@@ -1,39 +1,35 @@
 // Local SCD solver with block look-ahead: the same result as walking a partition's visiting order coordinate by
 // coordinate (paper Sec. 2.2 worker structure with L = 1; Sec. 5.1: SCD local solver), up to rounding order, with
-// the work that does not depend on earlier steps taken off the sequential chain.
+// everything that does not depend on the step before taken off the sequential chain.
 //
-// The walk is cut into blocks of 32 consecutive steps. Inside a block, with w the local model at the block's start,
-//     dot_j = x_j . w + sigma' * sum_{l < j} delta_l * (x_j . x_l),
-// so once the 32 dot products against w and the strictly lower triangle of the block's Gram matrix G_jl = x_j . x_l
-// are known, the 32 steps are a scalar recurrence run by one warp: a step costs the scalar map and a few fused
-// multiply-adds, plus one shuffle per coordinate to hand the results round. The block then applies
-// w += sigma' * sum_j delta_j x_j in parallel. Which coordinates meet in a block is fixed by the visiting order
-// alone, not by the model, so everything structural is prepared for all blocks of all partitions at once by a
-// throughput kernel that uses the whole GPU, and the latency-bound kernel (one CTA per partition) only consumes it.
+// The walk is cut into blocks of 32 consecutive steps. With w the local model some steps back,
+//     dot_j = x_j . w + sigma' * sum over the steps l since then of delta_l * (x_j . x_l),
+// so once the dot products against an OLDER model and the Gram entries x_j . x_l are known, the steps are a scalar
+// recurrence. A block's dot products are taken against the model as it was two blocks earlier (while the block
+// before it is still being walked); what the block before contributes comes from the cross Gram matrix of the two
+// blocks, what the block's own earlier steps contribute from its Gram triangle. Only the recurrence is sequential:
+// one warp runs it block after block without waiting for a model update, while the other warps, and the other CTAs
+// of the partition's thread-block cluster, apply block b's update to the model and take block b + 2's dot products.
 //
-//   k_lookahead_prepare   one CTA per block. Writes the block's record, one contiguous piece of memory: per-step
-//                         headers (coordinate, constants of the scalar step), the scaled Gram triangle, the block's
-//                         non-zeros packed row after row, and, for the entry ids that several coordinates of the
-//                         block share, the transposed view ("which non-zeros touch id i": one list per shared id,
-//                         in ascending coordinate order). An id that only one coordinate has is updated straight
-//                         from that coordinate's row; a shared id by a few threads that add up its list in a fixed
-//                         order: no atomics on the model, the same bits every run. Built with a shared-memory hash
-//                         table whose slots carry a 32-bit membership mask; a non-zero's place in its list is the
-//                         number of lower mask bits, so the lists need no sort and come out the same whatever order
-//                         the threads ran in.
-//   k_lookahead_chain     one CTA per partition, 16 warps. Per block: (G) all warps gather the dot products against
-//                         the local model; (R) warp 0 runs the recurrence while warp 1 starts the bulk copy of the
-//                         next block's record; (S) all threads apply the update. Entry ids below HOT (ids are
-//                         frequency-ranked) live in shared memory for the whole kernel as w = v + sigma' U_k; the
-//                         others are read from and added to row k of the update workspace in global memory.
+//   k_lookahead_prepare   one CTA per block; nothing in it depends on the model. Writes the block's records: for
+//                         the recurrence warp the per-step constants, the scaled Gram triangle and the scaled cross
+//                         Gram matrix with the next block; for each CTA of the cluster the block's non-zeros whose
+//                         entry id falls to that CTA (id mod cluster size), packed row after row, and for the ids
+//                         that several coordinates of the block share the transposed view (one list per id, in
+//                         ascending coordinate order), so that the model update needs no atomics and gives the same
+//                         bits every run.
+//   k_lookahead_chain     one cluster of C CTAs per partition. Entry ids below C * HOT (ids are frequency-ranked)
+//                         live in shared memory for the whole kernel as w = v + sigma' U_k, id i in CTA i mod C;
+//                         the others are read from and added to row k of the update workspace in global memory.
+//                         Warp 0 of CTA 0 runs the recurrence. The worker warps of every CTA loop over
+//                         "wait for block b's deltas, apply them to my part of the model, take my part of block
+//                         b + 2's dot products, send the 32 partial sums to CTA 0". Deltas and partial sums travel
+//                         through distributed shared memory by asynchronous stores that complete on the receiver's
+//                         mbarrier; no multicast, every wait bounded.
 //
-// A record arrives by ONE bulk copy. Measured: fetching the 32 coordinates straight from the matrix with two small
-// bulk copies each slowed whatever phase ran while those 64 copies landed by about 3 000 cycles per block (the
-// slow phase moved with the point of issue), three times what the recurrence itself costs.
-//
-// A block with a coordinate longer than 128 entries does not fit the shared-memory buffers: the prepare kernel
-// flags it and warp 0 walks it coordinate by coordinate. Rounds that span several local
-// epochs revisit coordinates, whose state the headers would not know: those take the blocked solver instead.
+// A block with more non-zeros than the shared-memory buffers hold is flagged by the prepare kernel: the pipeline
+// drains, warp 0 of CTA 0 walks the block coordinate by coordinate against the whole model, and the pipeline starts
+// again behind it. Rounds that span several local epochs run the pair of kernels once per epoch.
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -45,61 +41,80 @@ namespace chicle {
 
 namespace {
 
-constexpr int kLB = 32;          // steps per block
-constexpr int kCapL = 128;       // longest coordinate a staged block can hold
-constexpr int kMaxNz = kLB * kCapL;
-constexpr int kHT = 4096;        // slots of the prepare kernel's hash table (>= kMaxNz)
-constexpr int kPreThreads = 256;  // dense prepare kernel
-constexpr int kPreThreadsS = 512; // sparse prepare kernel
+constexpr int kLB = 32;            // steps per block
+constexpr int kMaxC = 8;           // CTAs per cluster at most (the portable limit)
+constexpr int kCapL = 128;         // longest dense coordinate
+constexpr int kIdBits = 26;        // entry ids of a staged non-zero (problems with more ids take the blocked solver)
+constexpr uint32_t kIdMask = (1u << kIdBits) - 1u;
 constexpr int kChainThreads = 512;
-constexpr int kChainWarps = kChainThreads / 32;
-constexpr int kRowsPerWarp = kLB / kChainWarps;
+constexpr int kSubSlots = 4;       // worker records in shared memory: blocks b .. b + 3
+constexpr int kHeadSlots = 3;      // recurrence records in shared memory
+// Worker warps: all but the warps that share warp 0's scheduler (warp ids 0, 4, 8, 12), which stay out of its way.
+constexpr int kWorkWarps = 12;
+constexpr int kWorkThreads = kWorkWarps * 32;
+constexpr int kBarWork = 1;        // named barrier of the worker warps
 
-struct alignas(16) LookHdr {
-    int64_t row_start;
+// Per-step constants for the recurrence warp (see coordinate_step for p0 .. p3).
+struct alignas(16) CHdr {
     int32_t coord;
-    int32_t nnz;
-    float p0, p1, p2, p3; // the constants of the scalar step (see coordinate_step)
-    float q0;             // what the states of the block's earlier coordinates at round start contribute (see below)
-    float pad[3];         // [0]: log of p2 for the logistic loss (the start of its Newton iteration needs it)
+    float p0, p1, p2, p3;
+    float A, B; // the recurrence's state starts at A + B * (dot product against the older model) (+ the cross terms)
+    float lq;   // logistic: log of p2
 };
-static_assert(sizeof(LookHdr) == 48, "header size");
+static_assert(sizeof(CHdr) == 32, "header size");
 
-// A block's record starts with this; behind it (sparse): val[total] f32, idx[total] i32 (the non-zeros row after row;
-// the top bit of idx marks an id that more than one coordinate of the block has), ids[T] i32 (those shared ids),
-// cpos[total] u16 (for a non-zero with a shared id: its place in the id's list; the lists lie one after the other,
-// each in ascending coordinate order), off[T + 1] u16 (where each list starts). Dense: val[cnt * dim].
-struct alignas(16) BlkHead {
-    int32_t T;         // entry ids that more than one coordinate of the block has
-    int32_t flags;     // bit 0: walk this block coordinate by coordinate (the record is the head alone)
-    int32_t cnt;       // steps in the block (32 but for a partition's last block)
-    int32_t total_nnz; // non-zeros of the block
-    uint16_t roff[kLB + 8]; // where each coordinate's non-zeros start in val / idx ([32] = total)
-    LookHdr hdr[kLB];
-    float G[kLB * kLB]; // G[l * 32 + j]: the scaled Gram entry of coordinates l < j (see below), else 0
+// What the recurrence warp reads for one block.
+struct alignas(16) ChainHead {
+    int32_t cnt;    // steps in the block (32 but for a partition's last block)
+    int32_t flags;  // bit 0: walk this block coordinate by coordinate
+    int32_t pad[2];
+    CHdr hdr[kLB];
+    float q0n[kLB];      // what the states of this block's coordinates at round start contribute to the next block
+    float G[kLB * kLB];  // G[l * 32 + j]: scaled Gram entry of this block's coordinates l < j, else 0
+    float X[kLB * kLB];  // X[l * 32 + j]: scaled Gram entry of this block's l with the NEXT block's j (0: no carry)
 };
-static_assert(sizeof(BlkHead) % 16 == 0, "bulk copy size");
+static_assert(sizeof(ChainHead) % 16 == 0, "bulk copy size");
 
-__host__ __device__ constexpr uint32_t record_bytes(int total, int T, bool dense)
+// What one CTA's workers read for one block. Behind it (sparse): val[n] f32, meta[n] u32 (entry id in the low bits,
+// the coordinate's place in the block above them, the top bit marks an id that several coordinates of the block
+// have), ids[T] u32 (those shared ids), cpos[n] u16 (for a non-zero with a shared id: its place in the id's list;
+// the lists lie one after the other, each in ascending coordinate order), off[T + 1] u16 (where each list starts).
+// Dense: val[cnt * dim].
+struct alignas(16) SubHead {
+    int32_t n;     // non-zeros of the block that fall to this CTA
+    int32_t T;     // shared ids among them
+    int32_t cnt;
+    int32_t flags; // bit 0 as in ChainHead (the record is then this head alone)
+    uint16_t roff[kLB + 8]; // where each coordinate's non-zeros start ([32] = n)
+};
+static_assert(sizeof(SubHead) == 96, "sub-record head");
+
+__host__ __device__ constexpr uint32_t sub_bytes(int n, int T, bool dense)
 {
-    return ((uint32_t)sizeof(BlkHead) + (dense ? 4u * total : 8u * total + 4u * T + 2u * total + 2u * (T + 1)) + 15u) & ~15u;
+    return ((uint32_t)sizeof(SubHead) + (dense ? 4u * n : 8u * n + 4u * T + 2u * n + 2u * (T + 1)) + 15u) & ~15u;
 }
 
-struct alignas(16) BlkDir { // where a block's record is
-    unsigned long long offset; // bytes from the start of the record buffer (a multiple of 16)
-    uint32_t bytes;            // a multiple of 16; 0: the record buffer was full
-    uint32_t pad;
+struct alignas(16) BlkDir { // where a record is
+    unsigned long long offset; // bytes from the start of the launch's region of the record buffer (a multiple of 16)
+    uint32_t bytes;            // a multiple of 16; 0: no record was written
+    uint32_t flags;            // bit 0: the block is walked coordinate by coordinate
 };
 
 struct LookParams {
     SolverParams S;
-    unsigned char *rec;         // the records
-    BlkDir *dir;                // one per block
-    unsigned long long *cursor; // [0]: bytes of `rec` handed out so far this round
-    unsigned long long rec_cap; // bytes of `rec`
-    const int64_t *blk_base;    // K + 1: the first block of each partition in this round's numbering of the blocks
-    int32_t K;
+    unsigned char *rec;          // this launch's region of the record buffer
+    BlkDir *dirH;                // one per block: the recurrence warp's record
+    BlkDir *dirS;                // C per block: the workers' records
+    unsigned long long *cursor;  // bytes of the pool handed out so far in this launch
+    unsigned long long *timing;  // scratch words of a -DCHICLE_LA_TIMING build
+    unsigned long long pool_off; // the pool of worker records starts here (the heads lie before it, one per block)
+    unsigned long long pool_cap; // bytes of the pool
+    const int64_t *blk_base;     // K + 1: the first block of each partition in this launch's numbering of the blocks
+    int32_t K, logC;
+    int32_t nzcap;               // non-zeros a worker record holds at most
+    int32_t hotc;                // entry ids per CTA kept in shared memory
     int64_t n_blocks;
+    int64_t drop_block;          // test aid: this block's records are left unpublished (-1: none)
 };
 
 #ifdef CHICLE_LA_TIMING
@@ -109,7 +124,6 @@ struct LookParams {
 #endif
 
 __device__ __forceinline__ int64_t steps_of(const LookParams &P, int64_t k, int64_t nk) { return partition_steps(P.S, k, nk); }
-__device__ __forceinline__ int64_t block_base(const LookParams &P, int64_t k) { return P.blk_base[k]; }
 __device__ __forceinline__ void block_to_part(const LookParams &P, int64_t bid, int &k, int64_t &b)
 {
     int32_t lo = 0, hi = P.K; // blk_base[lo] <= bid < blk_base[hi] (partitions may differ in size)
@@ -122,28 +136,14 @@ __device__ __forceinline__ void block_to_part(const LookParams &P, int64_t bid, 
     b = bid - P.blk_base[lo];
 }
 
-// blk_base[k] = blocks of the partitions before k (one thread: K is small next to the work of a round)
-__global__ void k_block_bases(SolverParams S, int32_t K, int64_t *__restrict__ blk_base)
+// The constants of coordinate c's scalar step (see coordinate_step), and the line A + B * dot that the recurrence's
+// state starts from (what the block's earlier coordinates contribute at their round-start states is taken off A
+// once the Gram triangle is known).
+template <int LOSS> __device__ __forceinline__ CHdr make_hdr(const SolverParams &P, int32_t c)
 {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    int64_t run = 0;
-    for (int32_t k = 0; k < K; ++k) {
-        blk_base[k] = run;
-        const int64_t steps = partition_steps(S, k, S.part_off[k + 1] - S.part_off[k]);
-        run += (steps + kLB - 1) / kLB;
-    }
-    blk_base[K] = run;
-}
-
-// The constants of coordinate c's scalar step (see coordinate_step).
-template <int LOSS> __device__ __forceinline__ LookHdr make_hdr(const SolverParams &P, int32_t c, int64_t rs, int32_t nnz)
-{
-    LookHdr hd;
-    hd.q0 = 0.0f;
-    hd.pad[0] = hd.pad[1] = hd.pad[2] = 0.0f;
-    hd.row_start = rs;
+    CHdr hd;
     hd.coord = c;
-    hd.nnz = nnz;
+    hd.lq = 0.0f;
     const float s = P.sqnorm[c];
     const float al = P.alpha[c];
     if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
@@ -151,15 +151,24 @@ template <int LOSS> __device__ __forceinline__ LookHdr make_hdr(const SolverPara
         hd.p1 = al;
         hd.p2 = 1.0f / fmaf(P.sigma * s, P.inv_n, P.lambda);
         hd.p3 = P.lambda;
+        hd.A = P.lambda * al;
+        hd.B = P.inv_n;
     } else {
         const float y = P.labels[c];
         hd.p0 = y / P.lam_n;
         hd.p1 = y * al;
         hd.p3 = y;
-        if (LOSS == CHICLE_LOSS_HINGE_DUAL) hd.p2 = s > 0.0f ? P.lam_n / (P.sigma * s) : CUDART_INF_F;
-        else {
+        if (LOSS == CHICLE_LOSS_HINGE_DUAL) {
+            const bool zero = !(s > 0.0f);
+            hd.p2 = zero ? CUDART_INF_F : P.lam_n / (P.sigma * s);
+            // a + (1 - y dot / (lambda n)) * p2; a zero row goes to a' = 1 whatever the model is
+            hd.A = zero ? 2.0f : hd.p2 + hd.p1;
+            hd.B = zero ? 0.0f : -hd.p0 * hd.p2;
+        } else {
             hd.p2 = P.sigma * s / P.lam_n;
-            hd.pad[0] = hd.p2 > 0.0f ? logf(hd.p2) : -CUDART_INF_F; // log q, for the start of the Newton iteration
+            hd.lq = hd.p2 > 0.0f ? logf(hd.p2) : -CUDART_INF_F; // log q, for the start of the Newton iteration
+            hd.A = hd.p2 * hd.p1;
+            hd.B = -hd.p0;
         }
     }
     return hd;
@@ -186,69 +195,80 @@ __device__ __forceinline__ float ldca_if(const float *p, bool on)
 }
 
 // The recurrence in the form the chain runs it. Every loss keeps one number s_j per coordinate that is linear in the
-// dot product, a scalar map s -> out, and the update s_j += Ghat[l][j] * out_l for the later coordinates j > l:
+// dot product, a scalar map s -> out, and the update s_j += Ghat[l][j] * out_l for the later coordinates j:
 //   hinge     s = a + (1 - y dot / (lambda n)) * lambda n / (sigma' |x|^2), out = a' = clip(s, 0, 1)
 //   logistic  s = q a - y dot / (lambda n),                                  out = a' = sigmoid(root of z + q sigmoid(z) = s)
 //   ridge     s = dot / n + lambda w,                                       out = delta = -s / (sigma' |c|^2 / n + lambda)
-// With dot_j = m0_j + sigma' sum_{l<j} delta_l G_jl and delta_l = y_l (a'_l - a_l) this gives, for the dual losses,
-// Ghat[l][j] = c_j y_l G_jl with c_j = -sigma' p2_j y_j / (lambda n) (hinge; 0 for a zero row) or -sigma' y_j / (lambda n)
-// (logistic), and s_j starts at its value for m0_j minus q0_j = sum_{l<j} Ghat[l][j] a_l, so that the chain adds
-// Ghat * a'_l and not Ghat * (a'_l - a_l). Ridge: Ghat[l][j] = sigma' G_jl / n, q0 = 0. The prepare kernel stores Ghat
-// and q0; a step of the chain is then: the scalar map, one shuffle, one fused multiply-add.
-template <int LOSS> __device__ __forceinline__ float gram_scale(const LookHdr &h, float sigma, float inv_n)
+// With dot_j = (older dot)_j + sigma' sum_l delta_l G_jl and delta_l = y_l (a'_l - a_l) this gives, for the dual
+// losses, Ghat[l][j] = c_j y_l G_jl with c_j = -sigma' p2_j y_j / (lambda n) (hinge; 0 for a zero row) or
+// -sigma' y_j / (lambda n) (logistic), and s_j starts sum_l Ghat[l][j] a_l lower, so that the chain adds
+// Ghat * a'_l and not Ghat * (a'_l - a_l). Ridge: Ghat[l][j] = sigma' G_jl / n, nothing to take off. The prepare kernel
+// stores Ghat (inside a block and from a block to the next) and the sums; a step of the chain is then: the scalar
+// map, one shuffle per four coordinates, one fused multiply-add.
+template <int LOSS> __device__ __forceinline__ float gram_scale(const CHdr &h, float sigma, float inv_n)
 {
     if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) return sigma * inv_n;
     if (LOSS == CHICLE_LOSS_HINGE_DUAL) return h.p2 < CUDART_INF_F ? -sigma * h.p0 * h.p2 : 0.0f;
     return -sigma * h.p0;
 }
-template <int LOSS> __device__ __forceinline__ float recurrence_start(float m0, const LookHdr &h)
+template <int LOSS> __device__ __forceinline__ float recurrence_map(float s, float p2, float lq)
 {
-    if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) return fmaf(m0, h.p0, h.p3 * h.p1);
-    if (LOSS == CHICLE_LOSS_HINGE_DUAL) return fmaf(1.0f - m0 * h.p0, h.p2, h.p1) - h.q0;
-    return fmaf(h.p2, h.p1, -(m0 * h.p0)) - h.q0;
-}
-template <int LOSS> __device__ __forceinline__ float recurrence_map(float s, const LookHdr &h)
-{
-    if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) return -s * h.p2;
+    if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) return -s * p2;
     if (LOSS == CHICLE_LOSS_HINGE_DUAL) return __saturatef(s);
-    return logistic_root(s, h.p2, h.pad[0]);
+    return logistic_root(s, p2, lq);
 }
 
-__device__ __forceinline__ uint32_t hash_id(int32_t id) { return ((uint32_t)id * 2654435761u) >> 20; } // 12 bits
-
-// Hands out `bytes` of the record buffer; false when it is full (cannot happen for a buffer sized by
-// lookahead_workspace; checked all the same).
-__device__ __forceinline__ bool take_record(const LookParams &P, uint32_t bytes, unsigned long long &offset)
+// The most frequent ids (ids are frequency-ranked) are in most of a block's coordinates. Their part of the Gram
+// matrices is taken from dense 32 x kHD tiles; only the other entries are walked through the table. Table slot: the id itself below kHD, a hashed slot above.
+constexpr int kHD = 32;
+constexpr int kHDS = kHD + 4; // row stride of the tiles: 16-byte loads of consecutive rows fall on different banks
+template <int HT> __device__ __forceinline__ uint32_t home_slot(int32_t id)
 {
-    offset = atomicAdd(P.cursor, (unsigned long long)bytes);
-    return offset + bytes <= P.rec_cap;
+    return id < kHD ? (uint32_t)id : kHD + (((uint32_t)id * 2654435761u) >> 16) % (uint32_t)(HT - kHD);
 }
+template <int HT> __device__ __forceinline__ uint32_t next_slot(uint32_t p) { return p + 1 < (uint32_t)HT ? p + 1 : kHD; }
 
 // ------------------------------------------------------------------------------------------------ prepare
+constexpr int kScanVals = 1 + kMaxC;
+
 template <int NZ, int HT, int THREADS> struct PreShared {
-    int32_t idx[NZ];     // the block's non-zeros, row after row
+    int32_t idx[NZ];     // the block's non-zeros, row after row (later: the membership mask of the non-zero's id)
     float val[NZ];
-    uint16_t slot[NZ];   // table slot of each non-zero's id
-    int32_t key[HT];        // id in a table slot, -1 = empty
-    uint32_t mask[HT];      // bit j: coordinate j of the block has this id
-    uint16_t soff[HT];      // start of the slot's list
-    float lval[NZ];      // the values of the non-zeros with shared ids, list after list (for the Gram pass)
+    uint16_t slot[NZ];   // table slot of each non-zero's id (later: where the id's list of values starts)
+    int32_t key[HT];     // id in a table slot, -1 = empty
+    uint32_t mask[HT];   // bit j: coordinate j of the block has this id
+    uint16_t soff[HT];   // start of the slot's list in lval
+    uint16_t coff[HT];   // a shared id: start of its list among the lists of its CTA's record
+    float lval[NZ];      // the values of the block's non-zeros, one list per id, each in ascending coordinate order
     float G[kLB][kLB + 1];
+    float X[kLB][kLB + 1];
+    alignas(16) float Dc[kLB][kHDS]; // this block's entries with the kHD most frequent ids, dense
+    alignas(16) float Dn[kLB][kHDS]; // the next block's
+    CHdr hdr[kLB];
+    float q0n[kLB];
     int64_t rs[kLB];
     int32_t nnz[kLB];
     int32_t roff[kLB + 1];
-    uint32_t warp_tot[THREADS / 32];
+    uint16_t rc[kLB + 1][kMaxC]; // non-zeros of coordinate j that fall to CTA c; then where they start in c's record
+    uint32_t warp_tot[THREADS / 32][kScanVals];
     float gsc[kLB], ys[kLB], as[kLB]; // per coordinate: its Gram scale, and what multiplies / enters from the earlier ones
-    int32_t total, too_long;
-    uint32_t bytes;
-    unsigned long long offset;
+    float gscn[kLB];                  // the next block's coordinates: their Gram scales
+    int64_t nrs[kLB];
+    int32_t nnnz[kLB];
+    unsigned long long sub_off[kMaxC];
+    uint32_t sub_len[kMaxC];
+    int32_t subT[kMaxC];
+    int32_t ncls[kMaxC]; // the next block's non-zeros per CTA
+    int32_t total, slow, carry, ncnt;
 };
 
-// One block's record (all threads of the CTA; every return below is taken by all of them).
+// One block's records (all threads of the CTA; every return below is taken by all of them).
 template <int LOSS, int NZ, int HT, int THREADS>
 __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t bid, PreShared<NZ, HT, THREADS> &sh)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    constexpr int NW = THREADS / 32;
+    const int C = 1 << P.logC;
     int k;
     int64_t b;
     block_to_part(P, bid, k, b);
@@ -256,174 +276,341 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
     const int64_t off = P.S.part_off[k] + (P.S.first_k ? P.S.first_k[k] : 0); // of this launch's first step in the order
     const int64_t steps = steps_of(P, k, nk);
     const int cnt = (int)((steps - b * kLB) < kLB ? (steps - b * kLB) : kLB);
+    const int64_t left = steps - (b + 1) * kLB; // steps behind this block
+    const int ncnt = left <= 0 ? 0 : (left < kLB ? (int)left : kLB);
+    ChainHead &out = *reinterpret_cast<ChainHead *>(P.rec + (size_t)bid * sizeof(ChainHead));
 #ifdef CHICLE_LA_TIMING
     long long pt0 = clock64(), pt1 = 0;
-#define PRE_T(i) do { asm volatile("" ::: "memory"); pt1 = clock64(); if (tid == 0) atomicAdd(P.cursor + 16 + (i), (unsigned long long)(pt1 - pt0)); pt0 = pt1; asm volatile("" ::: "memory"); } while (0)
+#define PRE_T(i) do { asm volatile("" ::: "memory"); pt1 = clock64(); if (tid == 0) atomicAdd(P.timing + 16 + (i), (unsigned long long)(pt1 - pt0)); pt0 = pt1; asm volatile("" ::: "memory"); } while (0)
 #else
 #define PRE_T(i) do { } while (0)
 #endif
 
-    // ---- headers (kept in registers of warp 0 until the record's place is known)
-    LookHdr hd{0, 0, 0, 0.f, 0.f, 0.f, 0.f, 0.f, {0.f, 0.f, 0.f}};
+    // ---- headers: warp 0 this block's coordinates, warp 1 the next block's
     if (warp == 0) {
+        CHdr hd{0, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        int64_t rs = 0;
+        int32_t n = 0;
         if (lane < cnt) {
             const int32_t c = P.S.perm[off + b * kLB + lane];
-            const int64_t rs = P.S.indptr[c], re = P.S.indptr[c + 1];
-            hd = make_hdr<LOSS>(P.S, c, rs, (int32_t)(re - rs));
+            rs = P.S.indptr[c];
+            n = (int32_t)(P.S.indptr[c + 1] - rs);
+            hd = make_hdr<LOSS>(P.S, c);
         }
-        sh.rs[lane] = hd.row_start;
-        sh.nnz[lane] = hd.nnz;
+        sh.hdr[lane] = hd;
+        sh.rs[lane] = rs;
+        sh.nnz[lane] = n;
         sh.gsc[lane] = lane < cnt ? gram_scale<LOSS>(hd, P.S.sigma, P.S.inv_n) : 0.0f;
         sh.ys[lane] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? 1.0f : hd.p3;
         sh.as[lane] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? 0.0f : hd.p1;
-        const bool too_long = __any_sync(0xffffffffu, hd.nnz > kCapL);
-        int incl = too_long ? 0 : hd.nnz;
+        int incl = n;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int t = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += t;
         }
-        // (a block with more non-zeros than this variant's arrays hold is walked in place as well)
-        const bool over = too_long || __shfl_sync(0xffffffffu, incl, 31) > NZ;
-        sh.roff[lane] = over ? 0 : incl - hd.nnz;
+        const int tot = __shfl_sync(0xffffffffu, incl, 31);
+        const bool over = tot > NZ; // more non-zeros than this kernel's arrays hold: walked in place
+        sh.roff[lane] = over ? 0 : incl - n;
         if (lane == 31) {
             sh.roff[kLB] = over ? 0 : incl;
             sh.total = over ? 0 : incl;
-            sh.too_long = over ? 1 : 0;
+            sh.slow = over ? 1 : 0;
+        }
+    } else if (warp == 1) {
+        CHdr hd{0, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        int64_t rs = 0;
+        int32_t n = 0;
+        if (lane < ncnt) {
+            const int32_t c = P.S.perm[off + (b + 1) * kLB + lane];
+            rs = P.S.indptr[c];
+            n = (int32_t)(P.S.indptr[c + 1] - rs);
+            hd = make_hdr<LOSS>(P.S, c);
+        }
+        sh.nrs[lane] = rs;
+        sh.nnnz[lane] = n;
+        sh.gscn[lane] = lane < ncnt ? gram_scale<LOSS>(hd, P.S.sigma, P.S.inv_n) : 0.0f;
+        int tot = n;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+        if (lane == 0) {
+            sh.ncnt = ncnt;
+            sh.carry = (ncnt > 0 && tot <= NZ) ? 1 : 0; // (and both blocks must be staged: see below)
         }
     }
     for (int p = tid; p < HT; p += THREADS) {
         sh.key[p] = -1;
         sh.mask[p] = 0u;
     }
+    for (int p = tid; p < (kLB + 1) * kMaxC; p += THREADS) (&sh.rc[0][0])[p] = 0;
+    for (int p = tid; p < kLB * kHDS; p += THREADS) {
+        (&sh.Dc[0][0])[p] = 0.0f;
+        (&sh.Dn[0][0])[p] = 0.0f;
+    }
+    if (tid < kMaxC) sh.ncls[tid] = 0;
     __syncthreads();
     PRE_T(0);
     const int total = sh.total;
-    bool slow = sh.too_long != 0;
+    const bool slow = sh.slow != 0;
+    const bool carry = !slow && sh.carry != 0;
     if (!slow) {
-        // ---- the block's non-zeros into shared memory, every id into the table
-        for (int j = warp; j < cnt; j += THREADS / 32) {
+        // ---- the block's non-zeros into shared memory, every id into the table; how many fall to each CTA. The
+        //      first 128 entries of a coordinate are loaded before any is used.
+        for (int j = warp; j < cnt; j += NW) {
             const int n = sh.nnz[j], r0 = sh.roff[j];
             const int64_t rs = sh.rs[j];
-            int32_t ids4[kCapL / 32];
-            float vals4[kCapL / 32];
+            int per_class[kMaxC];
 #pragma unroll
-            for (int c = 0; c < kCapL / 32; ++c) { // all of the row's loads first
+            for (int c = 0; c < kMaxC; ++c) per_class[c] = 0;
+            int32_t ids4[4];
+            float vals4[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
                 const int e = lane + 32 * c;
                 ids4[c] = e < n ? P.S.indices[rs + e] : -1;
                 vals4[c] = e < n ? P.S.values[rs + e] : 0.0f;
             }
-#pragma unroll
-            for (int c = 0; c < kCapL / 32; ++c) {
-                const int e = lane + 32 * c;
-                if (e >= n) continue;
-                const int32_t id = ids4[c];
-                sh.idx[r0 + e] = id;
-                sh.val[r0 + e] = vals4[c];
-                uint32_t p = hash_id(id) & (HT - 1);
-                for (int probe = 0; probe < HT; ++probe) {
-                    int32_t seen = sh.key[p];
-                    if (seen == -1) {
-                        seen = atomicCAS(&sh.key[p], -1, id);
-                        if (seen == -1) break;
+            auto take = [&](int e, int32_t id, float x) {
+                const bool on = id >= 0;
+                if (on) {
+                    sh.idx[r0 + e] = id;
+                    sh.val[r0 + e] = x;
+                    uint32_t p = home_slot<HT>(id);
+                    if (id < kHD) {
+                        sh.key[p] = id;
+                        sh.Dc[j][id] = x;
+                    } else {
+                        for (int probe = 0; probe < HT; ++probe) {
+                            int32_t seen = sh.key[p];
+                            if (seen == -1) {
+                                seen = atomicCAS(&sh.key[p], -1, id);
+                                if (seen == -1) break;
+                            }
+                            if (seen == id) break;
+                            p = next_slot<HT>(p);
+                        }
                     }
-                    if (seen == id) break;
-                    p = (p + 1) & (HT - 1);
+                    atomicOr(&sh.mask[p], 1u << j);
+                    sh.slot[r0 + e] = (uint16_t)p;
                 }
-                atomicOr(&sh.mask[p], 1u << j);
-                sh.slot[r0 + e] = (uint16_t)p;
+#pragma unroll
+                for (int c = 0; c < kMaxC; ++c)
+                    if (c < C) per_class[c] += __popc(__ballot_sync(0xffffffffu, on && (id & (C - 1)) == c));
+            };
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (32 * c < n) take(lane + 32 * c, ids4[c], vals4[c]);
+            for (int e0 = 128; e0 < n; e0 += 32) {
+                const int e = e0 + lane;
+                take(e, e < n ? P.S.indices[rs + e] : -1, e < n ? P.S.values[rs + e] : 0.0f);
+            }
+            if (lane == 0) {
+#pragma unroll
+                for (int c = 0; c < kMaxC; ++c) sh.rc[j][c] = (uint16_t)per_class[c];
             }
         }
-        __syncthreads();
-    PRE_T(1);
     }
-    // ---- number the shared ids (those with more than one bit in their mask) and lay out their lists: thread t owns
-    //      slots t, t + 256, ...; its running counts (ids in the high half, list entries in the low half) follow those
-    //      of the threads before it
-    uint32_t mine = 0;
+    __syncthreads();
+    PRE_T(1);
+    // ---- number the ids: every id's list of values for the Gram passes (soff), and for the ids that more than one
+    //      coordinate has, their number and their list's start inside their CTA's record. Thread t owns slots t,
+    //      t + THREADS, ...; its running counts follow those of the threads before it. v[0]: list entries of all ids;
+    //      v[1 + c]: CTA c's shared ids in the high half, their list entries in the low half.
+    uint32_t v[kScanVals];
+#pragma unroll
+    for (int i = 0; i < kScanVals; ++i) v[i] = 0u;
     if (!slow)
         for (int p = tid; p < HT; p += THREADS) {
             const uint32_t m = sh.mask[p];
-            if (m & (m - 1u)) mine += (1u << 16) + (uint32_t)__popc(m);
-        }
-    uint32_t incl = mine;
+            if (m == 0u) continue;
+            const uint32_t pc = (uint32_t)__popc(m);
+            v[0] += pc;
+            if (m & (m - 1u)) {
+                const int c = sh.key[p] & (C - 1);
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
+                for (int i = 0; i < kMaxC; ++i)
+                    if (i == c) v[1 + i] += (1u << 16) + pc;
+            }
+        }
+    uint32_t run[kScanVals];
+#pragma unroll
+    for (int i = 0; i < kScanVals; ++i) {
+        uint32_t incl = v[i];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) sh.warp_tot[warp][i] = incl;
+        run[i] = incl - v[i];
     }
-    if (lane == 31) sh.warp_tot[warp] = incl;
+    // where each coordinate's non-zeros start in each CTA's record (warp 0, lane = coordinate)
+    if (warp == 0 && !slow) {
+#pragma unroll
+        for (int c = 0; c < kMaxC; ++c) {
+            const int mine = sh.rc[lane][c];
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            sh.rc[lane][c] = (uint16_t)(incl - mine);
+            if (lane == 31) sh.rc[kLB][c] = (uint16_t)incl;
+        }
+    }
     __syncthreads();
     PRE_T(2);
-    uint32_t run = incl - mine, all = 0;
-    for (int w2 = 0; w2 < THREADS / 32; ++w2) {
-        if (w2 < warp) run += sh.warp_tot[w2];
-        all += sh.warp_tot[w2];
+    uint32_t all[kScanVals];
+#pragma unroll
+    for (int i = 0; i < kScanVals; ++i) {
+        all[i] = 0u;
+        for (int w2 = 0; w2 < NW; ++w2) {
+            if (w2 < warp) run[i] += sh.warp_tot[w2][i];
+            all[i] += sh.warp_tot[w2][i];
+        }
     }
-    const int T = (int)(all >> 16), total_m = (int)(all & 0xffffu);
-    // ---- the record's place (a block that is walked in place needs the head alone)
+    // ---- the records' places: the head has its own (one per block); the workers' records come from the pool. A
+    //      block that the pool has no room for is walked in place like one that is too long.
     if (tid == 0) {
-        unsigned long long offset = 0;
-        uint32_t bytes = slow ? (uint32_t)sizeof(BlkHead) : record_bytes(total, T, false);
-        if (!take_record(P, bytes, offset)) { offset = 0; bytes = 0; } // the chain kernel reports it
-        sh.offset = offset;
-        sh.bytes = bytes;
-        BlkDir d;
-        d.offset = offset;
-        d.bytes = bytes;
-        d.pad = 0;
-        P.dir[bid] = d;
+        unsigned long long need = 0;
+        uint32_t len[kMaxC];
+#pragma unroll
+        for (int c = 0; c < kMaxC; ++c) {
+            len[c] = c < C ? sub_bytes(sh.rc[kLB][c], (int)(all[1 + c] >> 16), false) : 0u;
+            need += len[c];
+        }
+        unsigned long long at = 0;
+        int sl = sh.slow;
+#pragma unroll
+        for (int c = 0; c < kMaxC; ++c)
+            if (c < C && sh.rc[kLB][c] > P.nzcap) sl = 1; // more of them fall to one CTA than its record holds
+        if (!sl) {
+            at = atomicAdd(P.cursor, need);
+            if (at + need > P.pool_cap) sl = 2;
+        }
+        sh.slow = sl;
+#pragma unroll
+        for (int c = 0; c < kMaxC; ++c) {
+            if (c >= C) continue;
+            BlkDir d;
+            if (sl) { // nothing to stage: the workers copy the first bytes of the head instead
+                d.offset = (unsigned long long)bid * sizeof(ChainHead);
+                d.bytes = 16u;
+                d.flags = 1u;
+            } else {
+                d.offset = P.pool_off + at;
+                d.bytes = len[c];
+                d.flags = 0u;
+                sh.sub_off[c] = d.offset;
+                sh.sub_len[c] = len[c];
+                sh.subT[c] = (int32_t)(all[1 + c] >> 16);
+                at += len[c];
+            }
+            if (bid == P.drop_block) d.bytes = 0u;
+            P.dirS[bid * C + c] = d;
+        }
     }
     __syncthreads();
     PRE_T(3);
-    if (sh.bytes == 0) return;
-    unsigned char *rec = P.rec + sh.offset;
-    BlkHead &out = *reinterpret_cast<BlkHead *>(rec);
-    if (warp == 0) {
-        out.hdr[lane] = hd;
-        out.roff[lane] = (uint16_t)sh.roff[lane];
-        if (lane < 8) out.roff[kLB + lane] = (uint16_t)sh.roff[kLB];
-        if (lane == 0) {
-            out.T = T; out.flags = slow ? 1 : 0; out.cnt = cnt; out.total_nnz = total;
-        }
+    const bool walk = sh.slow != 0; // (slow, or no room in the pool)
+    if (warp == 0 && lane == 0) {
+        out.cnt = cnt;
+        out.flags = walk ? 1 : 0;
+        out.pad[0] = out.pad[1] = 0;
     }
-    if (slow) return; // the rest of the head is not read for such a block
-    float *val_g = reinterpret_cast<float *>(rec + sizeof(BlkHead));
-    int32_t *idx_g = reinterpret_cast<int32_t *>(val_g + total);
-    int32_t *ids_g = idx_g + total;
-    uint16_t *cpos_g = reinterpret_cast<uint16_t *>(ids_g + T);
-    uint16_t *off_g = cpos_g + total;
+    if (walk) {
+        // the head carries the constants of the steps and nothing else; nothing is carried to the next block
+        if (warp == 0) {
+            out.hdr[lane] = sh.hdr[lane];
+            out.q0n[lane] = 0.0f;
+        }
+        for (int i = tid; i < kLB * kLB; i += THREADS) out.X[i] = 0.0f;
+        return;
+    }
+    // ---- the workers' record heads, shared-id tables and list starts
+    if (tid < C) {
+        SubHead &h = *reinterpret_cast<SubHead *>(P.rec + sh.sub_off[tid]);
+        h.n = sh.rc[kLB][tid];
+        h.T = sh.subT[tid];
+        h.cnt = cnt;
+        h.flags = 0;
+    }
+    for (int i = tid; i < C * (kLB + 8); i += THREADS) {
+        const int c = i / (kLB + 8), j = i - c * (kLB + 8);
+        reinterpret_cast<SubHead *>(P.rec + sh.sub_off[c])->roff[j] = sh.rc[j < kLB ? j : kLB][c];
+    }
     for (int p = tid; p < HT; p += THREADS) {
         const uint32_t m = sh.mask[p];
+        if (m == 0u) continue;
+        const uint32_t pc = (uint32_t)__popc(m);
+        sh.soff[p] = (uint16_t)run[0];
+        run[0] += pc;
         if (m & (m - 1u)) {
-            const uint32_t t = run >> 16, o = run & 0xffffu;
-            ids_g[t] = sh.key[p];
+            const int32_t id = sh.key[p];
+            const int c = id & (C - 1);
+            uint32_t r = 0u;
+#pragma unroll
+            for (int i = 0; i < kMaxC; ++i)
+                if (i == c) { r = run[1 + i]; run[1 + i] += (1u << 16) + pc; }
+            const uint32_t t = r >> 16, o = r & 0xffffu;
+            unsigned char *rec = P.rec + sh.sub_off[c];
+            const int n_c = sh.rc[kLB][c], T_c = sh.subT[c];
+            uint32_t *ids_g = reinterpret_cast<uint32_t *>(rec + sizeof(SubHead) + 8u * n_c);
+            uint16_t *off_g = reinterpret_cast<uint16_t *>(rec + sizeof(SubHead) + 8u * n_c + 4u * T_c + 2u * n_c);
+            ids_g[t] = (uint32_t)id;
             off_g[t] = (uint16_t)o;
-            sh.soff[p] = (uint16_t)o;
-            run += (1u << 16) + (uint32_t)__popc(m);
+            if ((int)t == T_c - 1) off_g[T_c] = (uint16_t)(o + pc);
+            sh.coff[p] = (uint16_t)o;
         }
     }
-    if (tid == 0) off_g[T] = (uint16_t)total_m;
+    if (tid < C && sh.subT[tid] == 0) { // no shared ids: the list of starts is its end alone
+        unsigned char *rec = P.rec + sh.sub_off[tid];
+        const int n_c = sh.rc[kLB][tid];
+        reinterpret_cast<uint16_t *>(rec + sizeof(SubHead) + 8u * n_c + 2u * n_c)[0] = 0;
+    }
     __syncthreads();
     PRE_T(4);
-    // ---- list entries: a non-zero's place in its id's list is the number of lower coordinates that have the id
-    for (int j = warp; j < cnt; j += THREADS / 32) {
+    // ---- the non-zeros into the workers' records, row after row: place = start of (coordinate, CTA) + rank among
+    //      the coordinate's non-zeros of that CTA; a shared id's place in its list is the number of lower
+    //      coordinates that have the id
+    for (int j = warp; j < cnt; j += NW) {
         const int n = sh.nnz[j], r0 = sh.roff[j];
-        for (int e = lane; e < n; e += 32) {
+        int before[kMaxC];
+#pragma unroll
+        for (int c = 0; c < kMaxC; ++c) before[c] = sh.rc[j][c];
+        for (int e0 = 0; e0 < n; e0 += 32) {
+            const int e = e0 + lane;
+            const bool on = e < n;
+            const int32_t id = on ? sh.idx[r0 + e] : 0;
+            const int cls = id & (C - 1);
+            int place = 0;
+#pragma unroll
+            for (int c = 0; c < kMaxC; ++c) {
+                if (c >= C) continue;
+                const uint32_t bal = __ballot_sync(0xffffffffu, on && cls == c);
+                if (cls == c) place = before[c] + __popc(bal & ((1u << lane) - 1u));
+                before[c] += __popc(bal);
+            }
+            if (!on) continue;
             const int p = sh.slot[r0 + e];
             const uint32_t m = sh.mask[p];
             const bool shared_id = (m & (m - 1u)) != 0u;
-            int pos = 0;
-            if (shared_id) {
-                pos = sh.soff[p] + __popc(m & ((1u << j) - 1u));
-                sh.lval[pos] = sh.val[r0 + e];
-            }
-            val_g[r0 + e] = sh.val[r0 + e];
-            idx_g[r0 + e] = sh.idx[r0 + e] | (shared_id ? (int32_t)0x80000000 : 0);
-            cpos_g[r0 + e] = (uint16_t)pos;
-            // for the Gram pass: the id itself is no longer needed, its mask and its list's start are
+            const int lower = __popc(m & ((1u << j) - 1u));
+            const float x = sh.val[r0 + e];
+            sh.lval[sh.soff[p] + lower] = x;
+            unsigned char *rec = P.rec + sh.sub_off[cls];
+            const int n_c = sh.rc[kLB][cls], T_c = sh.subT[cls];
+            float *val_g = reinterpret_cast<float *>(rec + sizeof(SubHead));
+            uint32_t *meta_g = reinterpret_cast<uint32_t *>(rec + sizeof(SubHead) + 4u * n_c);
+            uint16_t *cpos_g = reinterpret_cast<uint16_t *>(rec + sizeof(SubHead) + 8u * n_c + 4u * T_c);
+            val_g[place] = x;
+            meta_g[place] = (uint32_t)id | ((uint32_t)j << kIdBits) | (shared_id ? 0x80000000u : 0u);
+            cpos_g[place] = shared_id ? (uint16_t)(sh.coff[p] + lower) : (uint16_t)0;
+            // for the Gram pass: the id itself is no longer needed, its mask and its list's start are (top bit: one of
+            // the ids that the dense tiles cover)
             sh.idx[r0 + e] = (int32_t)m;
-            sh.slot[r0 + e] = sh.soff[p];
+            sh.slot[r0 + e] = (uint16_t)(sh.soff[p] | (id < kHD ? 0x8000 : 0));
         }
     }
     __syncthreads();
@@ -431,12 +618,20 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
     // ---- Gram triangle: a warp per coordinate j, lane l collects x_j . x_l over j's entries in ascending order. The
     //      lanes first look at 32 entries at once and keep those whose id an earlier coordinate has too; only these
     //      are then walked, their mask, list start and value handed round by shuffles.
-    for (int j = warp; j < kLB; j += THREADS / 32) {
+    for (int j = warp; j < kLB; j += NW) {
         float acc = 0.0f;
         if (j < cnt) {
             const int n = sh.nnz[j], r0 = sh.roff[j];
             const uint32_t below = (1u << j) - 1u, lt = (1u << lane) - 1u;
-            const bool mine = lane < j;
+            {
+                const float4 *dj = reinterpret_cast<const float4 *>(&sh.Dc[j][0]);
+                const float4 *dm = reinterpret_cast<const float4 *>(&sh.Dc[lane][0]);
+#pragma unroll
+                for (int h = 0; h < kHD / 4; ++h) {
+                    const float4 a = dj[h], b4 = dm[h];
+                    acc = fmaf(a.x, b4.x, acc); acc = fmaf(a.y, b4.y, acc); acc = fmaf(a.z, b4.z, acc); acc = fmaf(a.w, b4.w, acc);
+                }
+            }
             for (int e0 = 0; e0 < n; e0 += 32) {
                 const int e = e0 + lane;
                 uint32_t m_l = 0u;
@@ -447,7 +642,7 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
                     so_l = sh.slot[r0 + e];
                     x_l = sh.val[r0 + e];
                 }
-                uint32_t todo = __ballot_sync(0xffffffffu, (m_l & below) != 0u);
+                uint32_t todo = __ballot_sync(0xffffffffu, (m_l & below) != 0u && !(so_l & 0x8000)); // (not the dense ones)
                 // two entries per turn, so that the second one's loads are under way while the first is added
                 while (todo) {
                     const int src0 = __ffs(todo) - 1;
@@ -464,26 +659,121 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
                     acc = fmaf(x1, on1 ? v1 : 0.0f, acc);
                 }
             }
-            if (!mine) acc = 0.0f;
+            if (lane >= j) acc = 0.0f;
         }
         acc *= sh.gsc[j] * sh.ys[lane];
         sh.G[lane][j] = acc; // row l, column j
         float q0 = acc * sh.as[lane];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) q0 += __shfl_xor_sync(0xffffffffu, q0, o);
-        if (lane == 0 && j < cnt) out.hdr[j].q0 = q0;
+        if (lane == 0) sh.hdr[j].A -= q0;
+    }
+    PRE_T(6);
+    // ---- cross Gram matrix with the next block: a warp per coordinate j of the next block, whose non-zeros come
+    //      straight from the matrix and are looked up in this block's table; lane l collects x_j . x_l
+    for (int j = warp; j < kLB; j += NW) {
+        float acc = 0.0f;
+        if (carry && j < sh.ncnt) {
+            const int n = sh.nnnz[j];
+            const int64_t rs = sh.nrs[j];
+            const uint32_t lt = (1u << lane) - 1u;
+            int per_class[kMaxC];
+#pragma unroll
+            for (int c = 0; c < kMaxC; ++c) per_class[c] = 0;
+            int32_t ids4[4];
+            float vals4[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { // the first 128 entries are loaded before any is used
+                const int e = lane + 32 * c;
+                ids4[c] = e < n ? P.S.indices[rs + e] : -1;
+                vals4[c] = e < n ? P.S.values[rs + e] : 0.0f;
+            }
+            auto take = [&](int32_t id, float x_l) {
+                uint32_t m_l = 0u;
+                int so_l = 0;
+#pragma unroll
+                for (int c = 0; c < kMaxC; ++c)
+                    if (c < C) per_class[c] += __popc(__ballot_sync(0xffffffffu, id >= 0 && (id & (C - 1)) == c));
+                if (id >= 0 && id < kHD) sh.Dn[j][id] = x_l;
+                else if (id >= 0) {
+                    uint32_t p = home_slot<HT>(id);
+                    for (int probe = 0; probe < HT; ++probe) {
+                        const int32_t seen = sh.key[p];
+                        if (seen == id) { m_l = sh.mask[p]; so_l = sh.soff[p]; break; }
+                        if (seen == -1) break;
+                        p = next_slot<HT>(p);
+                    }
+                }
+                uint32_t todo = __ballot_sync(0xffffffffu, m_l != 0u);
+                while (todo) {
+                    const int src0 = __ffs(todo) - 1;
+                    todo &= todo - 1u;
+                    const bool two = todo != 0u;
+                    const int src1 = two ? __ffs(todo) - 1 : src0;
+                    todo &= todo - 1u;
+                    const uint32_t m0 = __shfl_sync(0xffffffffu, m_l, src0), m1 = __shfl_sync(0xffffffffu, m_l, src1);
+                    const int so0 = __shfl_sync(0xffffffffu, so_l, src0), so1 = __shfl_sync(0xffffffffu, so_l, src1);
+                    const float x0 = __shfl_sync(0xffffffffu, x_l, src0), x1 = __shfl_sync(0xffffffffu, x_l, src1);
+                    const bool on0 = (m0 >> lane) & 1u, on1 = two && ((m1 >> lane) & 1u);
+                    const float v0 = sh.lval[on0 ? so0 + __popc(m0 & lt) : 0], v1 = sh.lval[on1 ? so1 + __popc(m1 & lt) : 0];
+                    acc = fmaf(x0, on0 ? v0 : 0.0f, acc);
+                    acc = fmaf(x1, on1 ? v1 : 0.0f, acc);
+                }
+            };
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (32 * c < n) take(ids4[c], vals4[c]);
+            for (int e0 = 128; e0 < n; e0 += 32) {
+                const int e = e0 + lane;
+                take(e < n ? P.S.indices[rs + e] : -1, e < n ? P.S.values[rs + e] : 0.0f);
+            }
+            __syncwarp();
+            {
+                const float4 *dj = reinterpret_cast<const float4 *>(&sh.Dn[j][0]);
+                const float4 *dm = reinterpret_cast<const float4 *>(&sh.Dc[lane][0]);
+#pragma unroll
+                for (int h = 0; h < kHD / 4; ++h) {
+                    const float4 a = dj[h], b4 = dm[h];
+                    acc = fmaf(a.x, b4.x, acc); acc = fmaf(a.y, b4.y, acc); acc = fmaf(a.z, b4.z, acc); acc = fmaf(a.w, b4.w, acc);
+                }
+            }
+            if (lane >= cnt) acc = 0.0f;
+            if (lane == 0) {
+#pragma unroll
+                for (int c = 0; c < kMaxC; ++c)
+                    if (c < C && per_class[c]) atomicAdd(&sh.ncls[c], per_class[c]);
+            }
+        }
+        acc *= sh.gscn[j] * sh.ys[lane];
+        sh.X[lane][j] = acc; // row l (this block), column j (next block)
+        float q0 = acc * sh.as[lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) q0 += __shfl_xor_sync(0xffffffffu, q0, o);
+        if (lane == 0) sh.q0n[j] = q0;
     }
     __syncthreads();
-    PRE_T(6);
-    for (int i = tid; i < kLB * kLB; i += THREADS) out.G[i] = sh.G[i >> 5][i & 31];
     PRE_T(7);
+    // (a next block that is walked in place because more of its non-zeros fall to one CTA than a record holds takes
+    // nothing over either)
+    bool keep = true;
+#pragma unroll
+    for (int c = 0; c < kMaxC; ++c)
+        if (c < C && sh.ncls[c] > P.nzcap) keep = false;
+    for (int i = tid; i < kLB * kLB; i += THREADS) {
+        out.G[i] = sh.G[i >> 5][i & 31];
+        out.X[i] = keep ? sh.X[i >> 5][i & 31] : 0.0f;
+    }
+    if (warp == 0) {
+        out.hdr[lane] = sh.hdr[lane];
+        out.q0n[lane] = keep ? sh.q0n[lane] : 0.0f;
+    }
 }
 
 // A CTA takes blocks blockIdx.x, blockIdx.x + gridDim.x, ...: one each when the grid has a CTA per block; a launch
 // beside the chain kernels gets a grid that fits the SMs they leave, so that it never has CTAs waiting for an SM (which
 // would take the SMs of a finished chain launch before the next chain launch's CTAs, which need a whole SM each).
 template <int LOSS, int NZ, int HT, int THREADS>
-__global__ void __launch_bounds__(THREADS, 1024 / THREADS) k_lookahead_prepare(const LookParams P)
+__global__ void __launch_bounds__(THREADS) k_lookahead_prepare(const LookParams P)
 {
     extern __shared__ __align__(16) unsigned char smem_pre[];
     using Shared = PreShared<NZ, HT, THREADS>;
@@ -494,17 +784,22 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) k_lookahead_prepare(c
     }
 }
 
-// Short dense rows: every row has every id, so the lists are implicit: headers, Gram triangle and the rows.
+// Short dense rows: every row has every id, so the lists are implicit: constants, Gram triangle, cross Gram matrix
+// and the rows themselves (one worker record: the model lives in one CTA).
+constexpr int kPreThreads = 256;
 struct PreDenseShared {
-    float row[kLB][kCapL + 1];
-    float gsc[kLB], ys[kLB], as[kLB];
+    float row[2 * kLB][kCapL + 1]; // this block's rows, then the next block's
+    CHdr hdr[kLB];
+    float gsc[kLB], ys[kLB], as[kLB], gscn[kLB];
     unsigned long long offset;
     uint32_t bytes;
+    int32_t walk;
 };
 
 template <int LOSS> __device__ __forceinline__ void prepare_block_dense(const LookParams &P, const int64_t bid, PreDenseShared &sh)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    constexpr int NW = kPreThreads / 32;
     int k;
     int64_t b;
     block_to_part(P, bid, k, b);
@@ -512,66 +807,93 @@ template <int LOSS> __device__ __forceinline__ void prepare_block_dense(const Lo
     const int64_t off = P.S.part_off[k] + (P.S.first_k ? P.S.first_k[k] : 0); // of this launch's first step in the order
     const int64_t steps = steps_of(P, k, nk);
     const int cnt = (int)((steps - b * kLB) < kLB ? (steps - b * kLB) : kLB);
+    const int64_t left = steps - (b + 1) * kLB;
+    const int ncnt = left <= 0 ? 0 : (left < kLB ? (int)left : kLB);
     const int dim = (int)P.S.dim;
+    ChainHead &out = *reinterpret_cast<ChainHead *>(P.rec + (size_t)bid * sizeof(ChainHead));
     if (tid == 0) {
-        unsigned long long offset = 0;
-        uint32_t bytes = record_bytes(cnt * dim, 0, true);
-        if (!take_record(P, bytes, offset)) { offset = 0; bytes = 0; }
-        sh.offset = offset;
-        sh.bytes = bytes;
+        const uint32_t bytes = sub_bytes(cnt * dim, 0, true);
+        unsigned long long at = atomicAdd(P.cursor, (unsigned long long)bytes);
         BlkDir d;
-        d.offset = offset;
-        d.bytes = bytes;
-        d.pad = 0;
-        P.dir[bid] = d;
+        if (at + bytes > P.pool_cap) { // no room: walked in place
+            d.offset = (unsigned long long)bid * sizeof(ChainHead);
+            d.bytes = 16u;
+            d.flags = 1u;
+            sh.walk = 1;
+        } else {
+            d.offset = P.pool_off + at;
+            d.bytes = bytes;
+            d.flags = 0u;
+            sh.walk = 0;
+        }
+        sh.offset = d.offset;
+        if (bid == P.drop_block) d.bytes = 0u;
+        P.dirS[bid] = d;
+        out.cnt = cnt;
+        out.flags = sh.walk;
+        out.pad[0] = out.pad[1] = 0;
     }
     __syncthreads();
-    if (sh.bytes == 0) return;
+    const bool walk = sh.walk != 0;
     unsigned char *rec = P.rec + sh.offset;
-    BlkHead &out = *reinterpret_cast<BlkHead *>(rec);
-    float *val_g = reinterpret_cast<float *>(rec + sizeof(BlkHead));
-    for (int j = warp; j < kLB; j += kPreThreads / 32) {
+    float *val_g = reinterpret_cast<float *>(rec + sizeof(SubHead));
+    if (!walk && tid == 0) {
+        SubHead &h = *reinterpret_cast<SubHead *>(rec);
+        h.n = cnt * dim; h.T = 0; h.cnt = cnt; h.flags = 0;
+    }
+    if (!walk && tid < kLB + 8) reinterpret_cast<SubHead *>(rec)->roff[tid] = (uint16_t)((tid < cnt ? tid : cnt) * dim);
+    for (int j = warp; j < 2 * kLB; j += NW) {
+        const bool next = j >= kLB;
+        const int jj = next ? j - kLB : j;
+        const bool on = jj < (next ? ncnt : cnt);
         int32_t c = 0;
-        if (j < cnt) c = P.S.perm[off + b * kLB + j];
+        if (on) c = P.S.perm[off + (b + (next ? 1 : 0)) * kLB + jj];
         const int64_t rs = (int64_t)c * dim;
         for (int e = lane; e < dim; e += 32) {
-            const float x = j < cnt ? P.S.values[rs + e] : 0.0f;
+            const float x = on ? P.S.values[rs + e] : 0.0f;
             sh.row[j][e] = x;
-            if (j < cnt) val_g[j * dim + e] = x;
+            if (on && !next && !walk) val_g[jj * dim + e] = x;
         }
         if (lane == 0) {
-            LookHdr hd{0, 0, 0, 0.f, 0.f, 0.f, 0.f, 0.f, {0.f, 0.f, 0.f}};
-            if (j < cnt) hd = make_hdr<LOSS>(P.S, c, rs, dim);
-            out.hdr[j] = hd;
-            out.roff[j] = (uint16_t)((j < cnt ? j : cnt) * dim);
-            sh.gsc[j] = j < cnt ? gram_scale<LOSS>(hd, P.S.sigma, P.S.inv_n) : 0.0f;
-            sh.ys[j] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? 1.0f : hd.p3;
-            sh.as[j] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? 0.0f : hd.p1;
+            CHdr hd{0, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            if (on) hd = make_hdr<LOSS>(P.S, c);
+            const float gs = on ? gram_scale<LOSS>(hd, P.S.sigma, P.S.inv_n) : 0.0f;
+            if (next) sh.gscn[jj] = gs;
+            else {
+                sh.hdr[jj] = hd;
+                sh.gsc[jj] = gs;
+                sh.ys[jj] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? 1.0f : hd.p3;
+                sh.as[jj] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? 0.0f : hd.p1;
+            }
         }
     }
-    if (tid < 8) out.roff[kLB + tid] = (uint16_t)(cnt * dim);
-    if (tid == 0) {
-        out.T = dim; out.flags = 0; out.cnt = cnt; out.total_nnz = cnt * dim;
-    }
     __syncthreads();
-    // a warp per coordinate j, lane l has x_j . x_l
-    for (int j = warp; j < kLB; j += kPreThreads / 32) {
+    // a warp per column j; lane l has x_j . x_l: first inside the block (l < j), then from this block to the next
+    for (int j = warp; j < 2 * kLB; j += NW) {
+        const bool next = j >= kLB;
+        const int jj = next ? j - kLB : j;
         float acc = 0.0f;
-        if (lane < j)
+        if (!walk && (next ? lane < cnt : lane < jj))
             for (int e = 0; e < dim; ++e) acc = fmaf(sh.row[j][e], sh.row[lane][e], acc);
-        acc *= sh.gsc[j] * sh.ys[lane];
-        out.G[lane * kLB + j] = acc;
+        acc *= (next ? sh.gscn[jj] : sh.gsc[jj]) * sh.ys[lane];
+        (next ? out.X : out.G)[lane * kLB + jj] = acc;
         float q0 = acc * sh.as[lane];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) q0 += __shfl_xor_sync(0xffffffffu, q0, o);
-        if (lane == 0 && j < cnt) out.hdr[j].q0 = q0;
+        if (lane == 0) {
+            if (next) out.q0n[jj] = q0;
+            else sh.hdr[jj].A -= q0;
+        }
     }
+    __syncthreads();
+    if (tid < kLB) out.hdr[tid] = sh.hdr[tid];
 }
 
 // (blocks blockIdx.x, blockIdx.x + gridDim.x, ...: see k_lookahead_prepare)
 template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_prepare_dense(const LookParams P)
 {
-    __shared__ PreDenseShared sh;
+    extern __shared__ __align__(16) unsigned char smem_pre[];
+    PreDenseShared &sh = *reinterpret_cast<PreDenseShared *>(smem_pre);
     for (int64_t bid = blockIdx.x; bid < P.n_blocks; bid += gridDim.x) {
         prepare_block_dense<LOSS>(P, bid, sh);
         __syncthreads();
@@ -579,112 +901,261 @@ template <int LOSS> __global__ void __launch_bounds__(kPreThreads) k_lookahead_p
 }
 
 // ------------------------------------------------------------------------------------------------ chain
-template <bool DENSE, int HOT, int TMAX> struct ChainShared {
-    static constexpr uint32_t kRecMax = record_bytes(kMaxNz, DENSE ? 0 : TMAX, DENSE);
-    alignas(16) float W[HOT];                  // the local model v + sigma' U_k at the ids below HOT
-    alignas(16) unsigned char rec[2][kRecMax]; // the records of two consecutive blocks
-    alignas(8) uint64_t full[2];               // count the bytes of the bulk copies into rec[0] / rec[1]
-    float m0[kLB];                             // the block's dot products against the model at its start
-    float dj[kLB];                             // the block's deltas
-    float prod[DENSE ? 4 : kMaxNz];            // delta_j * x of the non-zeros with shared ids, list after list
-    float sink[32];                            // where a lane's stores go that have no target
+// Cluster plumbing. Addresses in another CTA's shared memory come from mapa; data and the signal that it has landed
+// travel together: an asynchronous store completes bytes on the receiver's mbarrier (no multicast anywhere).
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// Data and the signal that it has landed travel together: an asynchronous store completes bytes on the receiver's
+// mbarrier, straight from registers.
+__device__ __forceinline__ void st_async_f32(uint32_t remote, float v, uint32_t remote_bar)
+{
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(remote), "f"(v), "r"(remote_bar)
+                 : "memory");
+}
+__device__ __forceinline__ void st_async_f32x4_if(uint32_t remote, float a, float b, float c, float d, uint32_t remote_bar, bool on)
+{
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %6, 0;\n\t"
+                 "@q st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];\n\t}" ::"r"(remote),
+                 "f"(a), "f"(b), "f"(c), "f"(d), "r"(remote_bar), "r"((uint32_t)on)
+                 : "memory");
+}
+// Operations of a single lane as predicated instructions, not branches: a warp whose lanes part ways before a loop
+// of shuffles may run the loop as separate groups of lanes that meet again at every shuffle (measured: 125 cycles per
+// shuffle instead of 30 in the recurrence warp).
+__device__ __forceinline__ void bulk_g2s_if(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, bool on)
+{
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %4, 0;\n\t"
+                 "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar), "r"((uint32_t)on)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_if(uint32_t bar, uint32_t bytes, bool on)
+{
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}" ::"r"(bar),
+                 "r"(bytes), "r"((uint32_t)on)
+                 : "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t remote)
+{
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t remote, float v)
+{
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote_release(uint32_t remote_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+// One look at an mbarrier; the hardware may suspend the thread for up to `hint_ns` until the phase completes. The data
+// that the pipeline's barriers guard is written into this CTA's shared memory by asynchronous stores and copies that
+// complete on the barrier itself, so the default scope serves (as for a bulk copy); the two waits of the rare
+// walked-in-place path, which order ordinary stores of another CTA, add a cluster-scope fence of their own.
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t a, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(a), "r"(parity), "r"(100000u)
+        : "memory");
+    return ok;
+}
+// Bounded wait of one warp on an mbarrier that another CTA of the cluster completes (every lane must call it). No
+// pauses of its own (try_wait suspends the thread for a while by itself; the waits of the pipeline are short and on
+// its critical path); gives up after about a second, or when the CTA is aborting. The result is the same on all
+// lanes. One warp per CTA waits this way at a time.
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status)
+{
+    // every lane looks at the barrier (one instruction for the warp either way) and the lanes agree by a vote, so
+    // that the warp stays together
+    if (__all_sync(0xffffffffu, mbar_try_wait_cluster(bar, parity) != 0u)) return true;
+    const unsigned long long t_start = global_ns();
+    for (;;) {
+        bool ok = false;
+        for (int it = 0; it < 64 && !ok; ++it) ok = __all_sync(0xffffffffu, mbar_try_wait_cluster(bar, parity) != 0u);
+        if (ok) return true;
+        const bool stop = __any_sync(0xffffffffu, *abort_flag != 0);
+        const bool late = __any_sync(0xffffffffu, global_ns() - t_start > 1000000000ull);
+        if (stop || late) {
+            if (!stop && (threadIdx.x & 31) == 0) {
+                *abort_flag = 1;
+                atomicOr(status, ST_WAIT_TIMEOUT);
+            }
+            __syncwarp();
+            return false;
+        }
+    }
+}
+// The worker warps' barrier, with a vote: all of them take the same decision after a wait.
+__device__ __forceinline__ bool work_bar_and(bool ok)
+{
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, %2, %3, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(r)
+                 : "r"((uint32_t)ok), "n"(kBarWork), "n"(kWorkThreads)
+                 : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ void work_bar()
+{
+    asm volatile("bar.sync %0, %1;" ::"n"(kBarWork), "n"(kWorkThreads) : "memory");
+}
+
+struct alignas(16) ChainCtl {
+    uint64_t subfull[kSubSlots];   // count the bytes of the bulk copies into the workers' record slots
+    uint64_t headfull[kHeadSlots]; // the same for the recurrence warp's records (CTA 0)
+    uint64_t pbar[2];              // CTA 0: the partial dot products of a block have arrived from all CTAs
+    uint64_t dbar[2];              // a block's deltas have arrived from CTA 0
+    uint64_t ackbar;               // CTA 0: every CTA has applied all updates (before a block is walked in place)
+    alignas(16) float pbuf[2][kMaxC][kLB];
+    alignas(16) float dbuf[2][kLB];
+    float sink[32]; // where a lane's stores go that have no target
     int abort_flag;
+    int done; // the CTA's workers are through (the warps with no role sleep until then)
 };
 
-template <int LOSS, bool DENSE, int HOT, int TMAX, int NCH>
+// Shared-memory layout of the chain kernel (sizes fixed at launch): control, recurrence records, worker records,
+// products, the CTA's part of the model.
+struct ChainLayout {
+    uint32_t heads, subs, sub_stride, prod, w, total;
+};
+__host__ __device__ inline ChainLayout chain_layout(int nzcap, int hotc, bool dense, int dim)
+{
+    ChainLayout L;
+    L.heads = (uint32_t)((sizeof(ChainCtl) + 127) & ~(size_t)127);
+    L.subs = L.heads + kHeadSlots * (uint32_t)sizeof(ChainHead);
+    L.sub_stride = dense ? sub_bytes(kLB * dim, 0, true) : sub_bytes(nzcap, nzcap / 2, false);
+    L.prod = L.subs + kSubSlots * L.sub_stride;
+    L.w = L.prod + 4u * (uint32_t)(dense ? kLB : nzcap);
+    L.total = L.w + 4u * (uint32_t)(hotc > 0 ? hotc : 4);
+    return L;
+}
+
+template <int LOSS, bool DENSE>
 __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const LookParams P)
 {
-    using Shared = ChainShared<DENSE, HOT, TMAX>;
     extern __shared__ __align__(128) unsigned char smem_chain[];
-    Shared &sh = *reinterpret_cast<Shared *>(smem_chain);
-    const int k = blockIdx.x;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const SolverParams &S = P.S;
+    const int logC = P.logC, C = 1 << logC;
+    const uint32_t crank = cluster_ctarank();
+    const int k = (int)(blockIdx.x >> logC);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const ChainLayout L = chain_layout(P.nzcap, P.hotc, DENSE, (int)S.dim);
+    ChainCtl &ctl = *reinterpret_cast<ChainCtl *>(smem_chain);
+    float *W = reinterpret_cast<float *>(smem_chain + L.w);
+    float *prod = reinterpret_cast<float *>(smem_chain + L.prod);
+    volatile int *abort_flag = &ctl.abort_flag;
 
     const int64_t nk = S.part_off[k + 1] - S.part_off[k];
     const int64_t steps = steps_of(P, k, nk);
-    const int64_t nblocks = (steps + kLB - 1) / kLB;
-    const int64_t bid0 = block_base(P, k);
+    const int64_t nb = (steps + kLB - 1) / kLB;
+    const int64_t bid0 = P.blk_base[k];
     float *Uk = S.U + (size_t)k * (size_t)S.dim;
-    const int hot_n = HOT < S.dim ? HOT : (int)S.dim;
     const float sigma = S.sigma;
-    const float inv_sigma = 1.0f / sigma;
-    volatile int *abort_flag = &sh.abort_flag;
+    // entry ids below hot_total live in shared memory: id g in CTA g mod C at place g / C
+    const int64_t hot_all = (int64_t)P.hotc << logC;
+    const uint32_t hot_total = (uint32_t)(hot_all < S.dim ? hot_all : S.dim);
+    const int hot_mine = hot_total > crank ? (int)((hot_total - crank + C - 1) >> logC) : 0;
 
     if (tid == 0) {
-        sh.abort_flag = 0;
-        mbar_init(smem_u32(&sh.full[0]), 1);
-        mbar_init(smem_u32(&sh.full[1]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    for (int i = tid; i < hot_n; i += kChainThreads) sh.W[i] = fmaf(sigma, Uk[i], S.vbase[i]);
-    __syncthreads();
-    if (nblocks == 0) return;
-
-    // ---- warp 1: where a block's record is, and the copy itself. The directory entry of block b + 2 is loaded while
-    //      block b runs and first looked at a block later (an unconditional load from a clamped address, so that
-    //      nothing has to wait for it at the point of issue).
-    auto load_dir = [&](int64_t blk, uint32_t (&d)[4]) {
-        const int64_t at = blk < nblocks ? blk : nblocks - 1;
-        asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];"
-                     : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
-                     : "l"(P.dir + (bid0 + at))
-                     : "memory");
-    };
-    auto issue = [&](int64_t blk, const uint32_t (&d)[4]) {
-        if (blk >= nblocks || lane != 0) return;
-        const uint32_t bar = smem_u32(&sh.full[blk & 1]);
-        // the buffer was last written by ordinary stores: order them before the copy engine's writes
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        const unsigned long long offset = ((unsigned long long)d[1] << 32) | d[0];
-        const uint32_t bytes = d[2] <= Shared::kRecMax ? d[2] : 0u;
-        if (bytes == 0) {
-            // no record (the prepare kernel ran out of room): nothing will arrive, say so now
-            atomicOr(S.status, ST_WAIT_TIMEOUT);
-            *abort_flag = 1;
-            return;
+        ctl.abort_flag = 0;
+        ctl.done = 0;
+        for (int i = 0; i < kSubSlots; ++i) mbar_init(smem_u32(&ctl.subfull[i]), 1);
+        for (int i = 0; i < kHeadSlots; ++i) mbar_init(smem_u32(&ctl.headfull[i]), 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&ctl.pbar[i]), 1);
+            mbar_init(smem_u32(&ctl.dbar[i]), 1);
         }
-        mbar_arrive_expect_tx(bar, bytes);
-        bulk_g2s(smem_u32(&sh.rec[blk & 1][0]), P.rec + offset, bytes, bar);
-    };
-    uint32_t next_dir[4] = {0u, 0u, 0u, 0u};
-    if (warp == 1) {
-        load_dir(0, next_dir);
-        issue(0, next_dir);
-        load_dir(1, next_dir);
+        mbar_init(smem_u32(&ctl.ackbar), (uint32_t)C);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // armed for the first two blocks before anybody can send
+        for (int i = 0; i < 2; ++i) {
+            mbar_arrive_expect_tx(smem_u32(&ctl.pbar[i]), (uint32_t)(C * kLB * 4));
+            mbar_arrive_expect_tx(smem_u32(&ctl.dbar[i]), (uint32_t)(kLB * 4));
+        }
     }
+    for (int l = tid; l < hot_mine; l += kChainThreads) {
+        const size_t g = ((size_t)l << logC) + crank;
+        W[l] = fmaf(sigma, Uk[g], S.vbase[g]);
+    }
+    __syncthreads();
+    cluster_arrive();
+    cluster_wait();
 
+    const bool is_chain = crank == 0 && warp == 0;
+    const bool is_worker = (warp & 3) != 0;
     bool aborted = false;
+
+    if (is_chain && nb > 0) {
+        // ============================== the recurrence warp =====================================================
+        const int q = lane & 7, rep = lane >> 3;
+        auto head_at = [&](int64_t blk) { return reinterpret_cast<const ChainHead *>(smem_chain + L.heads + (size_t)(blk % kHeadSlots) * sizeof(ChainHead)); };
+        auto issue_head = [&](int64_t blk) {
+            const bool on = blk < nb && lane == 0;
+            const int64_t at = blk < nb ? blk : nb - 1;
+            const uint32_t bar = smem_u32(&ctl.headfull[at % kHeadSlots]);
+            mbar_arrive_expect_tx_if(bar, (uint32_t)sizeof(ChainHead), on);
+            bulk_g2s_if(smem_u32(head_at(at)), P.rec + (size_t)(bid0 + at) * sizeof(ChainHead), (uint32_t)sizeof(ChainHead), bar, on);
+        };
+        for (int i = 0; i < kHeadSlots; ++i) issue_head(i);
+        // where the deltas go: the copy `rep` of lane q sends the lane's four values to CTAs rep and rep + 4
+        uint32_t d_dst[2], d_bar[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint32_t c = (uint32_t)(rep + 4 * i) & (uint32_t)(C - 1);
+            d_dst[i] = mapa_u32(smem_u32(&ctl.dbuf[0][4 * q]), c);
+            d_bar[i] = mapa_u32(smem_u32(&ctl.dbar[0]), c);
+        }
+        float xs[4] = {0.f, 0.f, 0.f, 0.f}; // what the block before contributes to this block's states
+        int64_t fp = 0, sc = 0;            // staged blocks and walked blocks so far
 #ifdef CHICLE_LA_TIMING
-    long long tw = 0, tg1 = 0, tg = 0, tr = 0, tp1 = 0, ts = 0, trw = 0, t0 = clock64(), t1 = 0;
+        long long tw = 0, tr = 0, te = 0, t0 = clock64(), t1 = 0;
 #endif
-    for (int64_t b = 0; b < nblocks; ++b) {
-        unsigned char *rec = &sh.rec[b & 1][0];
-        const BlkHead &H = *reinterpret_cast<const BlkHead *>(rec);
-        // block b's record must have landed (bounded wait); one decision for the whole CTA, and at the same time the
-        // barrier between block b-1's update of the model and block b's reads
-        int ok = mbar_wait(smem_u32(&sh.full[b & 1]), (uint32_t)(b >> 1) & 1u, abort_flag, S.status) ? 1 : 0;
-        ok = __syncthreads_and(ok);
-        if (!ok) { aborted = true; break; }
-        LA_T(tw);
-        const int cnt = H.cnt;
-        const bool slow = (H.flags & 1) != 0;
-        if (slow) {
-            if (warp == 1) {
-                issue(b + 1, next_dir);
-                load_dir(b + 2, next_dir);
-            }
-            if (warp == 0) {
-                // coordinate by coordinate against the model: ids below HOT in shared memory, the rest in row k of
-                // the update workspace
+        for (int64_t b = 0; b < nb; ++b) {
+            if (!mbar_wait_cluster(smem_u32(&ctl.headfull[b % kHeadSlots]), (uint32_t)(b / kHeadSlots) & 1u, abort_flag, S.status)) { aborted = true; break; }
+            const ChainHead &H = *head_at(b);
+            const int cnt = H.cnt;
+            const uint32_t par = (uint32_t)(b & 1);
+            if (H.flags & 1) {
+                // ---- walked in place: wait until every CTA has applied all earlier updates, then coordinate by
+                //      coordinate against the whole model (the other CTAs' parts through the cluster's shared memory)
+                if (!mbar_wait_cluster(smem_u32(&ctl.ackbar), (uint32_t)sc & 1u, abort_flag, S.status)) { aborted = true; break; }
+                fence_cluster(); // the other CTAs' updates of their parts of the model, made by ordinary stores
+                ++sc;
+                const uint32_t w_base = smem_u32(W);
                 for (int j = 0; j < cnt; ++j) {
-                    const LookHdr h = H.hdr[j];
-                    const int32_t *ix = S.indices + h.row_start;
-                    const float *xv = S.values + h.row_start;
+                    const CHdr h = H.hdr[j];
+                    const int64_t rs = DENSE ? (int64_t)h.coord * S.dim : S.indptr[h.coord];
+                    const int n = DENSE ? (int)S.dim : (int)(S.indptr[h.coord + 1] - rs);
+                    const int32_t *ix = S.indices + rs;
+                    const float *xv = S.values + rs;
                     float acc = 0.0f, delta, new_state;
-                    for (int e = lane; e < h.nnz; e += 32) {
-                        const int32_t i = DENSE ? e : ix[e];
-                        const float ww = i < hot_n ? sh.W[i] : fmaf(sigma, __ldcg(Uk + i), S.vbase[i]);
+                    for (int e = lane; e < n; e += 32) {
+                        const uint32_t g = DENSE ? (uint32_t)e : (uint32_t)ix[e];
+                        const float ww = g < hot_total ? ld_cluster_f32(mapa_u32(w_base + 4u * (g >> logC), g & (uint32_t)(C - 1)))
+                                                       : fmaf(sigma, __ldcg(Uk + g), S.vbase[g]);
                         acc = fmaf(xv[e], ww, acc);
                     }
                     acc = warp_sum(acc);
@@ -695,325 +1166,461 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                         new_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? h.p1 : h.p3 * h.p1;
                     }
                     if (delta != 0.0f)
-                        for (int e = lane; e < h.nnz; e += 32) {
-                            const int32_t i = DENSE ? e : ix[e];
-                            if (i < hot_n) sh.W[i] = fmaf(sigma * delta, xv[e], sh.W[i]);
-                            else Uk[i] = fmaf(delta, xv[e], __ldcg(Uk + i));
+                        for (int e = lane; e < n; e += 32) {
+                            const uint32_t g = DENSE ? (uint32_t)e : (uint32_t)ix[e];
+                            if (g < hot_total) {
+                                const uint32_t a = mapa_u32(w_base + 4u * (g >> logC), g & (uint32_t)(C - 1));
+                                st_cluster_f32(a, fmaf(sigma * delta, xv[e], ld_cluster_f32(a)));
+                            } else Uk[g] = fmaf(delta, xv[e], __ldcg(Uk + g));
                         }
                     if (lane == 0) S.alpha[h.coord] = new_state;
                     __syncwarp();
                 }
-            }
-            continue;
-        }
-        const int total = H.total_nnz, T = H.T;
-        const float *val = reinterpret_cast<const float *>(rec + sizeof(BlkHead));
-        const int32_t *idx = reinterpret_cast<const int32_t *>(val + total);
-        const int32_t *ids = idx + total;
-        const uint16_t *cpos = reinterpret_cast<const uint16_t *>(ids + T);
-        const uint16_t *offs = cpos + total;
-        // ---------------- (G) dot products against the model at the block's start: warp w takes coordinates
-        //                  w and w + 16; all loads of the two are issued before anything is reduced
-        {
-            float acc[kRowsPerWarp];
-            int nn[kRowsPerWarp], r0[kRowsPerWarp];
+                // the walk's writes before the signal; the signal is a block of zero deltas
+                __threadfence();
+                fence_cluster();
+                __syncwarp();
 #pragma unroll
-            for (int r = 0; r < kRowsPerWarp; ++r) {
-                const int j = warp + kChainWarps * r;
-                r0[r] = H.roff[j] + lane;
-                nn[r] = H.roff[j + 1] - H.roff[j];
-                acc[r] = 0.0f;
-            }
-            int32_t id[kRowsPerWarp][NCH];
-            float x[kRowsPerWarp][NCH];
+                for (int i = 0; i < 2; ++i)
+                    st_async_f32x4_if(d_dst[i] + par * (uint32_t)(kLB * 4), 0.f, 0.f, 0.f, 0.f, d_bar[i] + par * 8u, rep + 4 * i < C);
+                xs[0] = xs[1] = xs[2] = xs[3] = 0.0f;
+            } else {
+                // ---- four coordinates at a time. Lane q (and its copies q + 8, q + 16, q + 24, which compute the
+                //      same) keeps the states of coordinates 4q .. 4q + 3. Group g: its lane walks its four coordinates
+                //      by itself, the four results are handed round, and every lane adds what they mean for its own
+                //      four, in this block and in the next.
+                float hp1[4], hp2[4], hp3[4], hlq[4], s[4], mine[4];
+                int32_t hcoord[4];
+                float hA[4], hB[4];
 #pragma unroll
-            for (int r = 0; r < kRowsPerWarp; ++r)
+                for (int i = 0; i < 4; ++i) {
+                    const CHdr &h = H.hdr[4 * q + i];
+                    hcoord[i] = h.coord; hp1[i] = h.p1; hp2[i] = h.p2; hp3[i] = h.p3; hlq[i] = h.lq; hA[i] = h.A; hB[i] = h.B;
+                    mine[i] = 0.0f;
+                }
+                const float4 q0n = *reinterpret_cast<const float4 *>(&H.q0n[4 * q]);
+                if (!mbar_wait_cluster(smem_u32(&ctl.pbar[fp & 1]), (uint32_t)(fp >> 1) & 1u, abort_flag, S.status)) { aborted = true; break; }
+                LA_T(tw);
+                float m0[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int c = 0; c < C; ++c) { // the CTAs' partial sums in a fixed order
+                    const float4 pv = *reinterpret_cast<const float4 *>(&ctl.pbuf[fp & 1][c][4 * q]);
+                    m0[0] += pv.x; m0[1] += pv.y; m0[2] += pv.z; m0[3] += pv.w;
+                }
+                __syncwarp();
 #pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const bool valid = lane + 32 * c < nn[r];
-                    id[r][c] = -1;
-                    x[r][c] = 0.0f;
-                    if (valid) {
-                        x[r][c] = val[r0[r] + 32 * c];
-                        id[r][c] = DENSE ? lane + 32 * c : (idx[r0[r] + 32 * c] & 0x7fffffff);
+                for (int i = 0; i < 4; ++i) s[i] = fmaf(hB[i], m0[i], hA[i]) + xs[i];
+                xs[0] = -q0n.x; xs[1] = -q0n.y; xs[2] = -q0n.z; xs[3] = -q0n.w;
+                const float4 *G4 = reinterpret_cast<const float4 *>(H.G); // G4[l * 8 + q]: row l, columns 4q .. 4q + 3
+                const float4 *X4 = reinterpret_cast<const float4 *>(H.X);
+#pragma unroll
+                for (int g = 0; g < kLB / 4; ++g) {
+                    float4 blk[4], nxt[4];
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        blk[kk] = G4[(4 * g + kk) * 8 + q];
+                        nxt[kk] = X4[(4 * g + kk) * 8 + q];
+                    }
+                    // inside the group (the numbers matter on the lanes with q == g, where blk holds the group's own
+                    // triangle; the others run the same instructions on copies)
+                    float o[4];
+                    o[0] = recurrence_map<LOSS>(s[0], hp2[0], hlq[0]);
+                    const float t1 = fmaf(o[0], blk[0].y, s[1]);
+                    o[1] = recurrence_map<LOSS>(t1, hp2[1], hlq[1]);
+                    const float t2 = fmaf(o[1], blk[1].z, fmaf(o[0], blk[0].z, s[2]));
+                    o[2] = recurrence_map<LOSS>(t2, hp2[2], hlq[2]);
+                    const float t3 = fmaf(o[2], blk[2].w, fmaf(o[1], blk[1].w, fmaf(o[0], blk[0].w, s[3])));
+                    o[3] = recurrence_map<LOSS>(t3, hp2[3], hlq[3]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mine[i] = q == g ? o[i] : mine[i];
+                    float og[4];
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) og[kk] = __shfl_sync(0xffffffffu, o[kk], g);
+                    // (zero entries of the triangle make this a no-op for the groups at or before g, whose states are final)
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        s[0] = fmaf(og[kk], blk[kk].x, s[0]);
+                        s[1] = fmaf(og[kk], blk[kk].y, s[1]);
+                        s[2] = fmaf(og[kk], blk[kk].z, s[2]);
+                        s[3] = fmaf(og[kk], blk[kk].w, s[3]);
+                        xs[0] = fmaf(og[kk], nxt[kk].x, xs[0]);
+                        xs[1] = fmaf(og[kk], nxt[kk].y, xs[1]);
+                        xs[2] = fmaf(og[kk], nxt[kk].z, xs[2]);
+                        xs[3] = fmaf(og[kk], nxt[kk].w, xs[3]);
                     }
                 }
-            // ids below HOT from shared memory; the others from row k of the update workspace (read at L2: the
-            // updates are made there by reductions) and from v, every load issued before any is used
-            float hv[kRowsPerWarp][NCH], uu[kRowsPerWarp][NCH], vb[kRowsPerWarp][NCH];
-#pragma unroll
-            for (int r = 0; r < kRowsPerWarp; ++r)
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const int32_t i = id[r][c];
-                    const bool cold = i >= hot_n;
-                    hv[r][c] = sh.W[(i >= 0 && !cold) ? i : 0];
-                    uu[r][c] = DENSE ? 0.0f : ldcg_if(Uk + (cold ? i : 0), cold);
-                    vb[r][c] = DENSE ? 0.0f : ldca_if(S.vbase + (cold ? i : 0), cold);
-                }
-#pragma unroll
-            for (int r = 0; r < kRowsPerWarp; ++r)
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const float ww = id[r][c] >= hot_n ? fmaf(sigma, uu[r][c], vb[r][c]) : hv[r][c];
-                    acc[r] = fmaf(x[r][c], ww, acc[r]); // x is 0 beyond the coordinate's length
-                }
-            if (NCH * 32 < kCapL) {
-#pragma unroll
-                for (int r = 0; r < kRowsPerWarp; ++r)
-                    for (int e = lane + 32 * NCH; e < nn[r]; e += 32) {
-                        const int a = r0[r] + e - lane;
-                        const int32_t i = DENSE ? e : (idx[a] & 0x7fffffff);
-                        const float ww = i < hot_n ? sh.W[i] : fmaf(sigma, __ldcg(Uk + i), S.vbase[i]);
-                        acc[r] = fmaf(val[a], ww, acc[r]);
-                    }
-            }
-            LA_T(tg1);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-                for (int r = 0; r < kRowsPerWarp; ++r) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
-            if (lane == 0) {
-#pragma unroll
-                for (int r = 0; r < kRowsPerWarp; ++r) sh.m0[warp + kChainWarps * r] = acc[r];
-            }
-        }
-        __syncthreads();
-        LA_T(tg);
-        // ---------------- (R) the recurrence on warp 0; warp 1 starts the next block's copy meanwhile
-        if (warp == 0) {
-            // Four coordinates at a time. Lane q (and its copies q + 8, q + 16, q + 24, which compute the same) keeps
-            // the states of coordinates 4q .. 4q + 3. Group g: its lane walks its four coordinates by itself (no
-            // shuffle inside a group), the four results are handed round, and every lane adds what they mean for
-            // its own four: the step per coordinate costs about half of one shuffle per coordinate.
-            const int q = lane & 7;
-            const float4 *G4 = reinterpret_cast<const float4 *>(H.G); // G4[l * 8 + q]: row l, columns 4q .. 4q + 3
-            LookHdr hh[4];
-            float s[4], mine[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                hh[i] = H.hdr[4 * q + i];
-                s[i] = recurrence_start<LOSS>(sh.m0[4 * q + i], hh[i]);
-                mine[i] = 0.0f;
-            }
-#pragma unroll
-            for (int g = 0; g < kLB / 4; ++g) {
-                float4 blk[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) blk[k] = G4[(4 * g + k) * 8 + q];
-                // inside the group (the numbers matter on the lanes with q == g, where blk holds the group's own
-                // triangle; the others run the same instructions on copies)
-                float o[4];
-                o[0] = recurrence_map<LOSS>(s[0], hh[0]);
-                const float t1 = fmaf(o[0], blk[0].y, s[1]);
-                o[1] = recurrence_map<LOSS>(t1, hh[1]);
-                const float t2 = fmaf(o[1], blk[1].z, fmaf(o[0], blk[0].z, s[2]));
-                o[2] = recurrence_map<LOSS>(t2, hh[2]);
-                const float t3 = fmaf(o[2], blk[2].w, fmaf(o[1], blk[1].w, fmaf(o[0], blk[0].w, s[3])));
-                o[3] = recurrence_map<LOSS>(t3, hh[3]);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) mine[i] = q == g ? o[i] : mine[i];
-                float og[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) og[k] = __shfl_sync(0xffffffffu, o[k], g);
-                // (zero entries of the triangle make this a no-op for the groups at or before g, whose states are final)
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    s[0] = fmaf(og[k], blk[k].x, s[0]);
-                    s[1] = fmaf(og[k], blk[k].y, s[1]);
-                    s[2] = fmaf(og[k], blk[k].z, s[2]);
-                    s[3] = fmaf(og[k], blk[k].w, s[3]);
-                }
-            }
-            if (lane < 8) {
+                LA_T(tr);
+                float dl[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int j = 4 * q + i;
-                    const LookHdr &h = hh[i];
                     float my_delta = 0.0f;
                     if (j < cnt) {
                         float my_state;
                         if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
                             my_delta = mine[i];
-                            my_state = h.p1 + mine[i];
+                            my_state = hp1[i] + mine[i];
                         } else {
-                            my_delta = h.p3 * (mine[i] - h.p1);
-                            my_state = h.p3 * mine[i];
+                            my_delta = hp3[i] * (mine[i] - hp1[i]);
+                            my_state = hp3[i] * mine[i];
                         }
                         if (!(fabsf(my_delta) <= CUDART_MAX_NORMAL_F)) {
                             atomicOr(S.status, ST_NONFINITE_STEP);
                             my_delta = 0.0f;
-                            my_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? h.p1 : h.p3 * h.p1;
+                            my_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? hp1[i] : hp3[i] * hp1[i];
                         }
-                        S.alpha[h.coord] = my_state;
+                        S.alpha[hcoord[i]] = my_state; // (the four copies of a lane store the same value)
                     }
-                    sh.dj[j] = my_delta;
+                    dl[i] = my_delta;
                 }
+                // armed for block fp + 2 before the deltas go out (its dot products are sent only after they arrive)
+                mbar_arrive_expect_tx_if(smem_u32(&ctl.pbar[fp & 1]), (uint32_t)(C * kLB * 4), lane == 0);
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+                    st_async_f32x4_if(d_dst[i] + par * (uint32_t)(kLB * 4), dl[0], dl[1], dl[2], dl[3], d_bar[i] + par * 8u, rep + 4 * i < C);
+                ++fp;
+                LA_T(te);
             }
-            LA_T(trw);
-        } else if (warp == 1) {
-            issue(b + 1, next_dir);
-            load_dir(b + 2, next_dir);
+            __syncwarp();
+            issue_head(b + kHeadSlots);
         }
-        __syncthreads();
-        LA_T(tr);
-        // ---------------- (S) the model update
-        if (DENSE) {
-            const int dim = (int)S.dim;
-            if (tid < dim) {
-                float sum = 0.0f;
-#pragma unroll 8
-                for (int j = 0; j < cnt; ++j) sum = fmaf(sh.dj[j], val[j * dim + tid], sum);
-                sh.W[tid] = fmaf(sigma, sum, sh.W[tid]);
-            }
-        } else {
-            // (A) row after row: a non-zero whose id no other coordinate of the block has is applied at once; the
-            //     others leave their product delta_j * x at their place in the id's list. No two of a thread's
-            //     non-zeros touch the same word, so all loads are issued before the first store.
-            {
-                int32_t i2[kRowsPerWarp][NCH];
-                float p2[kRowsPerWarp][NCH], w2[kRowsPerWarp][NCH];
-                int cp[kRowsPerWarp][NCH];
-                int a0[kRowsPerWarp], n2[kRowsPerWarp];
-                float d2[kRowsPerWarp];
-#pragma unroll
-                for (int r = 0; r < kRowsPerWarp; ++r) {
-                    const int j = warp + kChainWarps * r;
-                    a0[r] = H.roff[j] + lane;
-                    n2[r] = H.roff[j + 1] - H.roff[j];
-                    d2[r] = sh.dj[j];
-                }
-#pragma unroll
-                for (int r = 0; r < kRowsPerWarp; ++r)
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        const bool valid = lane + 32 * c < n2[r];
-                        const int a = valid ? a0[r] + 32 * c : 0;
-                        i2[r][c] = valid ? idx[a] : 0x7fffffff; // (an id beyond every range: nothing to do)
-                        p2[r][c] = d2[r] * val[a];
-                        cp[r][c] = cpos[a];
-                    }
-#pragma unroll
-                for (int r = 0; r < kRowsPerWarp; ++r)
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) w2[r][c] = sh.W[(i2[r][c] >= 0 && i2[r][c] < hot_n) ? i2[r][c] : 0];
-                // one store per non-zero, its address chosen without a branch: the list place, the model word, or a
-                // word of this lane's own that nobody reads; ids beyond HOT add to the workspace row instead
-                const uint32_t a_prod = smem_u32(&sh.prod[0]), a_w = smem_u32(&sh.W[0]), a_sink = smem_u32(&sh.sink[lane]);
-#pragma unroll
-                for (int r = 0; r < kRowsPerWarp; ++r)
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        const int32_t i = i2[r][c];
-                        const float p = p2[r][c];
-                        const uint32_t addr = i < 0 ? a_prod + 4u * (uint32_t)cp[r][c] : (i < hot_n ? a_w + 4u * (uint32_t)i : a_sink);
-                        sts_f32(addr, i < 0 ? p : fmaf(sigma, p, w2[r][c]));
-                        // a reduction at L2, nothing to wait for; one coordinate per id and block, blocks in order: a
-                        // fixed order of additions
-                        red_add_if(Uk + ((i >= hot_n && i != 0x7fffffff) ? i : 0), p, i >= hot_n && i != 0x7fffffff && p != 0.0f);
-                    }
-                if (NCH * 32 < kCapL) {
-#pragma unroll
-                    for (int r = 0; r < kRowsPerWarp; ++r)
-                        for (int e = lane + 32 * NCH; e < n2[r]; e += 32) {
-                            const int a = a0[r] + e - lane;
-                            const int32_t i = idx[a];
-                            const float p = d2[r] * val[a];
-                            if (i < 0) sh.prod[cpos[a]] = p;
-                            else if (i < hot_n) sh.W[i] = fmaf(sigma, p, sh.W[i]);
-                            else if (p != 0.0f) atomicAdd(Uk + i, p);
-                        }
-                }
-            }
-            LA_T(tp1);
-            __syncthreads();
-            // (B) four threads per shared id: each adds every fourth entry of the list (at most 8: a list has at most
-            //     32), then the four partial sums are added in a fixed order; two ids per thread and pass, all loads
-            //     first
-            const int quarter = tid & 3;
-            constexpr int kIdsPerPass = kChainThreads / 4;
-            for (int tb = 0; tb < T; tb += 2 * kIdsPerPass) {
-                float sum[2];
-                int32_t i3[2];
-                bool on[2];
-                int o0[2], o1[2];
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int t = tb + u * kIdsPerPass + (tid >> 2);
-                    on[u] = t < T;
-                    o0[u] = on[u] ? offs[t] + quarter : 0;
-                    o1[u] = on[u] ? offs[t + 1] : 0;
-                    i3[u] = on[u] ? ids[t] : 0;
-                }
-                float v[2][8];
-#pragma unroll
-                for (int u = 0; u < 2; ++u)
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const int o = o0[u] + 4 * q;
-                        v[u][q] = o < o1[u] ? sh.prod[o] : 0.0f;
-                    }
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    sum[u] = ((v[u][0] + v[u][1]) + (v[u][2] + v[u][3])) + ((v[u][4] + v[u][5]) + (v[u][6] + v[u][7]));
-                    sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 1);
-                    sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 2);
-                }
-#pragma unroll
-                for (int u = 0; u < 2; ++u)
-                    if (quarter == 0 && on[u] && sum[u] != 0.0f) {
-                        if (i3[u] < hot_n) sh.W[i3[u]] = fmaf(sigma, sum[u], sh.W[i3[u]]);
-                        else atomicAdd(Uk + i3[u], sum[u]);
-                    }
-            }
-        }
-        LA_T(ts);
-    }
 #ifdef CHICLE_LA_TIMING
-#ifndef LA_TIMING_TID
-#define LA_TIMING_TID 0
+        if (blockIdx.x == 0 && lane == 0) {
+            unsigned long long *d = P.timing;
+            d[0] = tw; d[1] = tr; d[2] = te; d[3] = nb;
+        }
 #endif
-    if (blockIdx.x == 0 && tid == LA_TIMING_TID) {
-        unsigned long long *d = P.cursor + 2;
-        d[0] = tw; d[1] = tg1; d[2] = tg; d[3] = tr; d[4] = tp1; d[5] = ts; d[6] = nblocks; d[7] = trw;
     }
+    if (is_worker && nb > 0) {
+        // ============================== the worker warps ========================================================
+        const int wt = (warp - 1 - (warp >> 2)) * 32 + lane; // 0 .. kWorkThreads - 1
+        const uint32_t p_bar0 = mapa_u32(smem_u32(&ctl.pbar[0]), 0u);
+        const uint32_t p_buf0 = mapa_u32(smem_u32(&ctl.pbuf[0][crank][0]), 0u);
+        const uint32_t ack_bar = mapa_u32(smem_u32(&ctl.ackbar), 0u);
+        const int dim = (int)S.dim;
+        auto sub_at = [&](int64_t blk) { return smem_chain + L.subs + (size_t)(blk & (kSubSlots - 1)) * L.sub_stride; };
+        // The directory entry of a block is loaded a block ahead of its use (an unconditional load from a clamped
+        // address, so that nothing has to wait for it at the point of issue).
+        auto load_dir = [&](int64_t blk, uint32_t (&d)[4]) {
+            const int64_t at = blk < nb ? blk : nb - 1;
+            asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+                         : "l"(P.dirS + (((bid0 + at) << logC) + crank))
+                         : "memory");
+        };
+        auto issue_sub = [&](int64_t blk, const uint32_t (&d)[4]) {
+            const uint32_t bar = smem_u32(&ctl.subfull[blk & (kSubSlots - 1)]);
+            // (the slot is only ever written by the copy engine and read by loads that are done by now)
+            const unsigned long long offset = ((unsigned long long)d[1] << 32) | d[0];
+            const uint32_t bytes = d[2] <= L.sub_stride ? d[2] : 0u;
+            const bool mine = blk < nb && wt == 0;
+            if (mine && bytes == 0) {
+                // no record: nothing will arrive, say so now
+                atomicOr(S.status, ST_WAIT_TIMEOUT);
+                *abort_flag = 1;
+            }
+            mbar_arrive_expect_tx_if(bar, bytes, mine && bytes != 0);
+            bulk_g2s_if(smem_u32(sub_at(blk)), P.rec + offset, bytes, bar, mine && bytes != 0);
+        };
+        // which of the blocks b .. b + 3 are walked in place
+        bool sl0, sl1, sl2, sl3;
+        {
+            uint32_t d[4];
+            load_dir(0, d); issue_sub(0, d); sl0 = (d[3] & 1u) != 0u;
+            load_dir(1, d); issue_sub(1, d); sl1 = nb > 1 && (d[3] & 1u) != 0u;
+            load_dir(2, d); issue_sub(2, d); sl2 = nb > 2 && (d[3] & 1u) != 0u;
+            load_dir(3, d); issue_sub(3, d); sl3 = nb > 3 && (d[3] & 1u) != 0u;
+        }
+        int64_t fg = 0; // staged blocks whose dot products have been sent
+#ifdef CHICLE_LA_TIMING
+        long long wd = 0, ws = 0, wg = 0, ws1 = 0, wg0 = 0, wg1 = 0, t0 = clock64(), t1 = 0;
 #endif
-    if (aborted) {
-        // the status word has the reason; give a copy that may still be in flight one more bounded wait, write nothing
-        (void)mbar_wait(smem_u32(&sh.full[0]), 0u, abort_flag, S.status);
-        return;
+
+        // Block x's dot products against the model as it is now (this CTA's part), sent to CTA 0.
+        auto take_dots = [&](int64_t x) -> bool {
+            bool ok = wt >= 32 || mbar_wait_cluster(smem_u32(&ctl.subfull[x & (kSubSlots - 1)]), (uint32_t)(x >> 2) & 1u, abort_flag, S.status);
+            ok = work_bar_and(ok); // (also: the products of the phase before have been read)
+            if (!ok) return false;
+            LA_T(wg0);
+            const unsigned char *rec = sub_at(x);
+            const SubHead &h = *reinterpret_cast<const SubHead *>(rec);
+            const float *val = reinterpret_cast<const float *>(rec + sizeof(SubHead));
+            const uint32_t slot = (uint32_t)(fg & 1);
+            if (DENSE) {
+                if (wt < kLB * 8) {
+                    const int j = wt >> 3, qq = wt & 7;
+                    float acc = 0.0f;
+                    if (j < h.cnt)
+                        for (int e = qq; e < dim; e += 8) acc = fmaf(val[j * dim + e], W[e], acc);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+                    if (qq == 0) prod[j] = acc;
+                }
+                work_bar();
+                if (wt < kLB) {
+                    st_async_f32(p_buf0 + (slot * (uint32_t)(kMaxC * kLB) + (uint32_t)wt) * 4u, prod[wt], p_bar0 + slot * 8u);
+                }
+            } else {
+                const int n = h.n;
+                const uint32_t *meta = reinterpret_cast<const uint32_t *>(val + n);
+                // Eight threads per coordinate, each its every eighth non-zero: the first two with all loads issued
+                // before anything is used. Ids below hot_total from shared memory; the others from row k of the
+                // update workspace (read at L2: the updates are made there by reductions) and from v.
+                if (wt < kLB * 8) {
+                    const int j = wt >> 3, qq = wt & 7;
+                    const int lo = h.roff[j] + qq, hi = h.roff[j + 1];
+                    float x[2], hv[2], uu[2], vb[2];
+                    bool cold[2];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int e = lo + 8 * u;
+                        const bool on = e < hi;
+                        x[u] = on ? val[e] : 0.0f;
+                        const uint32_t g = on ? (meta[e] & kIdMask) : 0u;
+                        cold[u] = on && g >= hot_total;
+                        hv[u] = W[cold[u] ? 0u : (g >> logC)];
+                        uu[u] = ldcg_if(Uk + (cold[u] ? g : 0u), cold[u]);
+                        vb[u] = ldca_if(S.vbase + (cold[u] ? g : 0u), cold[u]);
+                    }
+                    float acc = x[0] * (cold[0] ? fmaf(sigma, uu[0], vb[0]) : hv[0]);
+                    acc = fmaf(x[1], cold[1] ? fmaf(sigma, uu[1], vb[1]) : hv[1], acc);
+                    for (int e = lo + 16; e < hi; e += 8) {
+                        const uint32_t g = meta[e] & kIdMask;
+                        const float ww = g < hot_total ? W[g >> logC] : fmaf(sigma, __ldcg(Uk + g), S.vbase[g]);
+                        acc = fmaf(val[e], ww, acc);
+                    }
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+                    if (qq == 0) st_async_f32(p_buf0 + (slot * (uint32_t)(kMaxC * kLB) + (uint32_t)j) * 4u, acc, p_bar0 + slot * 8u);
+                }
+                LA_T(wg1);
+            }
+            ++fg;
+            return true;
+        };
+
+        if (!sl0) aborted = !take_dots(0);
+        if (!aborted && nb > 1 && !sl0 && !sl1) aborted = !take_dots(1);
+        LA_T(wg);
+        for (int64_t b = 0; b < nb && !aborted; ++b) {
+            uint32_t dn[4];
+            load_dir(b + kSubSlots, dn);
+            const uint32_t par = (uint32_t)(b & 1);
+            if (sl0) {
+                // walked in place by CTA 0: every update before it has been applied here (the barrier that ended
+                // the block before); say so, and wait for the walk to end
+                if (wt == 0) mbar_arrive_remote_release(ack_bar);
+                bool ok = wt >= 32 || mbar_wait_cluster(smem_u32(&ctl.dbar[par]), (uint32_t)(b >> 1) & 1u, abort_flag, S.status);
+                if (wt < 32) fence_cluster(); // the walk's ordinary stores into this CTA's part of the model
+                ok = work_bar_and(ok);
+                if (!ok) { aborted = true; break; }
+            } else {
+                bool ok = wt >= 32 || mbar_wait_cluster(smem_u32(&ctl.dbar[par]), (uint32_t)(b >> 1) & 1u, abort_flag, S.status);
+                ok = work_bar_and(ok);
+                if (!ok) { aborted = true; break; }
+                LA_T(wd);
+                // ---- block b's update of this CTA's part of the model
+                const float *dl = ctl.dbuf[par];
+                const unsigned char *rec = sub_at(b);
+                const SubHead &h = *reinterpret_cast<const SubHead *>(rec);
+                const float *val = reinterpret_cast<const float *>(rec + sizeof(SubHead));
+                if (DENSE) {
+                    if (wt < dim) {
+                        float sum = 0.0f;
+                        const int cnt = h.cnt;
+#pragma unroll 8
+                        for (int j = 0; j < cnt; ++j) sum = fmaf(dl[j], val[j * dim + wt], sum);
+                        W[wt] = fmaf(sigma, sum, W[wt]);
+                    }
+                } else {
+                    const int n = h.n, T = h.T;
+                    const uint32_t *meta = reinterpret_cast<const uint32_t *>(val + n);
+                    const uint32_t *ids = meta + n;
+                    const uint16_t *cpos = reinterpret_cast<const uint16_t *>(ids + T);
+                    const uint16_t *offs = cpos + n;
+                    // (A) eight threads per coordinate. A non-zero whose id no other coordinate of the block has is
+                    //     applied at once (no two of a block's non-zeros touch the same word then); the others leave
+                    //     their product delta_j * x at their place in the id's list. One store per non-zero, its
+                    //     address chosen without a branch: the list place, the model word, or a word that nobody reads;
+                    //     ids beyond the part in shared memory add to the workspace row instead.
+                    if (wt < kLB * 8) {
+                        const int j = wt >> 3, qq = wt & 7;
+                        const int lo = h.roff[j] + qq, hi = h.roff[j + 1];
+                        const float d = dl[j];
+                        const uint32_t a_prod = smem_u32(prod), a_w = smem_u32(W), a_sink = smem_u32(&ctl.sink[lane]);
+                        uint32_t m[2];
+                        float p[2], w2[2];
+                        int cp[2];
+                        bool on[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int e = lo + 8 * u;
+                            on[u] = e < hi;
+                            m[u] = on[u] ? meta[e] : 0u;
+                            p[u] = on[u] ? d * val[e] : 0.0f;
+                            cp[u] = on[u] ? cpos[e] : 0;
+                        }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const uint32_t g = m[u] & kIdMask;
+                            w2[u] = W[(on[u] && g < hot_total) ? (g >> logC) : 0u];
+                        }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const uint32_t g = m[u] & kIdMask;
+                            const bool shared_id = (m[u] >> 31) != 0u, hot = g < hot_total;
+                            const uint32_t addr = !on[u] ? a_sink : (shared_id ? a_prod + 4u * (uint32_t)cp[u] : (hot ? a_w + 4u * (g >> logC) : a_sink));
+                            sts_f32(addr, shared_id ? p[u] : fmaf(sigma, p[u], w2[u]));
+                            const bool far = on[u] && !shared_id && !hot && p[u] != 0.0f;
+                            red_add_if(Uk + (far ? g : 0u), p[u], far); // a reduction at L2, nothing waits for it
+                        }
+                        for (int e = lo + 16; e < hi; e += 8) {
+                            const uint32_t mm = meta[e];
+                            const uint32_t g = mm & kIdMask;
+                            const float pp = d * val[e];
+                            if (mm & 0x80000000u) prod[cpos[e]] = pp;
+                            else if (g < hot_total) W[g >> logC] = fmaf(sigma, pp, W[g >> logC]);
+                            else if (pp != 0.0f) atomicAdd(Uk + g, pp);
+                        }
+                    }
+                    work_bar();
+                    LA_T(ws1);
+                    // (B) four threads per shared id: each adds every fourth entry of the list (at most 8: a list has
+                    //     at most 32), then the four partial sums are added in a fixed order; two ids per thread and
+                    //     pass, all loads first
+                    const int quarter = wt & 3;
+                    constexpr int kIdsPerPass = kWorkThreads / 4;
+                    for (int tb = 0; tb < T; tb += 2 * kIdsPerPass) {
+                        float sum[2];
+                        uint32_t g3[2];
+                        bool on[2];
+                        int o0[2], o1[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int t = tb + u * kIdsPerPass + (wt >> 2);
+                            on[u] = t < T;
+                            o0[u] = on[u] ? offs[t] + quarter : 0;
+                            o1[u] = on[u] ? offs[t + 1] : 0;
+                            g3[u] = on[u] ? ids[t] : 0u;
+                        }
+                        float vv[2][8];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u)
+#pragma unroll
+                            for (int qq = 0; qq < 8; ++qq) {
+                                const int o = o0[u] + 4 * qq;
+                                vv[u][qq] = o < o1[u] ? prod[o] : 0.0f;
+                            }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            sum[u] = ((vv[u][0] + vv[u][1]) + (vv[u][2] + vv[u][3])) + ((vv[u][4] + vv[u][5]) + (vv[u][6] + vv[u][7]));
+                            sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 1);
+                            sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 2);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u)
+                            if (quarter == 0 && on[u] && sum[u] != 0.0f) {
+                                if (g3[u] < hot_total) W[g3[u] >> logC] = fmaf(sigma, sum[u], W[g3[u] >> logC]);
+                                else atomicAdd(Uk + g3[u], sum[u]);
+                            }
+                    }
+                }
+                work_bar();
+            }
+            mbar_arrive_expect_tx_if(smem_u32(&ctl.dbar[par]), (uint32_t)(kLB * 4), wt == 0); // for block b + 2
+            issue_sub(b + kSubSlots, dn); // block b's slot is free
+            LA_T(ws);
+            // a block right behind a walked one starts from the model as the walk left it
+            if (sl0 && b + 1 < nb && !sl1) {
+                if (!take_dots(b + 1)) { aborted = true; break; }
+            }
+            if (b + 2 < nb && !sl2 && !sl1) {
+                if (!take_dots(b + 2)) { aborted = true; break; }
+            }
+            sl0 = sl1; sl1 = sl2; sl2 = sl3;
+            sl3 = b + kSubSlots < nb && (dn[3] & 1u) != 0u;
+            LA_T(wg);
+        }
+#ifdef CHICLE_LA_TIMING
+        if (blockIdx.x == 0 && wt == 0) {
+            unsigned long long *d = P.timing + 4;
+            d[0] = wd; d[1] = ws; d[2] = wg; d[3] = ws1; d[4] = wg0; d[5] = wg1;
+        }
+#endif
+        if (!aborted) {
+            work_bar();
+            const float inv_sigma = 1.0f / sigma;
+            for (int l = wt; l < hot_mine; l += kWorkThreads) {
+                const size_t g = ((size_t)l << logC) + crank;
+                Uk[g] = (W[l] - S.vbase[g]) * inv_sigma;
+            }
+        }
     }
-    __syncthreads();
-    for (int i = tid; i < hot_n; i += kChainThreads) Uk[i] = (sh.W[i] - S.vbase[i]) * inv_sigma;
+    if (is_worker || nb == 0) {
+        if ((tid & 31) == 0) *reinterpret_cast<volatile int *>(&ctl.done) = 1;
+    } else if (!is_chain) {
+        // a warp with no role sleeps until the workers are through: waiting at the cluster barrier from the start
+        // would take issue slots from the recurrence warp, which shares its scheduler with these warps
+        const volatile int *done = &ctl.done;
+        for (uint32_t it = 0; it < (1u << 24) && !*done; ++it) __nanosleep(2000);
+    }
+    // nobody leaves while another CTA of the cluster may still write to, or read from, its shared memory
+    __syncwarp();
+    cluster_arrive();
+    cluster_wait();
 }
 
-constexpr int kHotSkew = 24064;
-constexpr int kTmax = kMaxNz / 2; // an id is shared by at least two of a block's non-zeros
-
-template <int LOSS, bool DENSE, int HOT, int TMAX, int NCH> cudaError_t launch_chain(Glm &g, const LookParams &P)
+// blk_base of every slice in one launch: slice s of partition k takes slice[(2s) K + k] steps
+__global__ void k_block_bases_slices(const int64_t *__restrict__ slice, int32_t K, int64_t *__restrict__ blk_base)
 {
-    using Shared = ChainShared<DENSE, HOT, TMAX>;
-    static_assert(sizeof(Shared) <= 227 * 1024, "shared memory budget");
-    auto kern = k_lookahead_chain<LOSS, DENSE, HOT, TMAX, NCH>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Shared));
+    if (threadIdx.x != 0) return;
+    const int s = blockIdx.x;
+    const int64_t *steps = slice + (size_t)s * 2 * (size_t)K;
+    int64_t *out = blk_base + (size_t)s * ((size_t)K + 1);
+    int64_t run = 0;
+    for (int32_t k = 0; k < K; ++k) {
+        out[k] = run;
+        run += (steps[k] + kLB - 1) / kLB;
+    }
+    out[K] = run;
+}
+
+template <int LOSS, bool DENSE> cudaError_t launch_chain(Glm &g, const LookParams &P)
+{
+    auto kern = k_lookahead_chain<LOSS, DENSE>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.la_smem);
     if (e != cudaSuccess) return e;
-    kern<<<g.K, kChainThreads, sizeof(Shared), g.stream>>>(P);
-    e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)g.K << g.la_logC, 1, 1);
+    cfg.blockDim = dim3(kChainThreads, 1, 1);
+    cfg.dynamicSmemBytes = g.la_smem;
+    cfg.stream = g.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1u << g.la_logC;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kern, P);
 #ifdef CHICLE_LA_TIMING
-    unsigned long long t[12] = {0};
-    (void)cudaStreamSynchronize(g.stream);
-    (void)cudaMemcpy(t, P.cursor + 2, sizeof(t), cudaMemcpyDeviceToHost);
-    const double nb = t[6] ? (double)t[6] : 1.0;
-    fprintf(stderr, "lookahead chain, cycles per block (CTA 0): wait %.0f gather %.0f reduce+bar %.0f recurrence %.0f products %.0f "
-            "lists %.0f (%llu blocks); warp 0's recurrence alone %.0f, then waiting for warp 1 %.0f\n", t[0] / nb, t[1] / nb, t[2] / nb,
-            (t[3] + t[7]) / nb, t[4] / nb, t[5] / nb, t[6], t[7] / nb, t[3] / nb);
+    if (e == cudaSuccess) {
+        unsigned long long t[12] = {0};
+        (void)cudaStreamSynchronize(g.stream);
+        (void)cudaMemcpy(t, P.timing, sizeof(t), cudaMemcpyDeviceToHost);
+        const double nb = t[3] ? (double)t[3] : 1.0;
+        fprintf(stderr, "lookahead chain, cycles per block (partition 0): waiting for dot products %.0f, recurrence %.0f, deltas %.0f; "
+                "workers of CTA 0: waiting for deltas %.0f, update: row-wise %.0f, lists and copy issue %.0f, dot products: record wait %.0f, "
+                "products %.0f, sums and sending %.0f (%llu blocks)\n",
+                t[0] / nb, t[1] / nb, t[2] / nb, t[4] / nb, t[7] / nb, t[5] / nb, t[8] / nb, t[9] / nb, t[6] / nb, t[3]);
+    }
 #endif
     return e;
 }
 
-template <int LOSS, int NZ, int HT, int THREADS> cudaError_t launch_prepare(Glm &g, const LookParams &P, unsigned nb, cudaStream_t stream)
+template <int LOSS, int NZ, int HT, int THREADS> cudaError_t launch_prepare(const LookParams &P, unsigned nb, cudaStream_t stream)
 {
-    (void)g;
     using Shared = PreShared<NZ, HT, THREADS>;
     auto pre = k_lookahead_prepare<LOSS, NZ, HT, THREADS>;
     cudaError_t e = cudaFuncSetAttribute(pre, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Shared));
@@ -1022,74 +1629,92 @@ template <int LOSS, int NZ, int HT, int THREADS> cudaError_t launch_prepare(Glm 
     return cudaGetLastError();
 }
 
+constexpr int kPreSmallNz = 2048;
+
+// true: the prepare kernel with arrays for 2 048 non-zeros per block serves (32 coordinates of 50 on average, with room)
+bool small_prepare(const Glm &g) { return 32.0 * (double)g.nnz / (double)g.n_coord * 1.25 <= (double)kPreSmallNz; }
+
 // The prepare kernel of one launch's blocks on `stream`.
 template <int LOSS> cudaError_t launch_prepare_on(Glm &g, const LookParams &P, cudaStream_t stream)
 {
     const unsigned nb = (unsigned)P.n_blocks;
+    if (nb == 0) return cudaSuccess;
     // beside the chain kernels: no more CTAs than fit the SMs the chains leave (see k_lookahead_prepare)
-    const unsigned free_sms = (unsigned)(g.sm_count > g.K ? g.sm_count - g.K : 1);
+    const int chain_sms = g.K << g.la_logC;
+    const unsigned free_sms = (unsigned)(g.sm_count > chain_sms ? g.sm_count - chain_sms : 1);
     if (g.fmt == CHICLE_FMT_DENSE_ROWMAJOR) {
-        const unsigned per_sm = 2048 / kPreThreads;
+        const unsigned per_sm = 4;
         const unsigned grid = stream == g.stream || nb < free_sms * per_sm ? nb : free_sms * per_sm;
-        k_lookahead_prepare_dense<LOSS><<<grid, kPreThreads, 0, stream>>>(P);
+        auto pre = k_lookahead_prepare_dense<LOSS>;
+        cudaError_t e = cudaFuncSetAttribute(pre, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PreDenseShared));
+        if (e != cudaSuccess) return e;
+        pre<<<grid, kPreThreads, sizeof(PreDenseShared), stream>>>(P);
         return cudaGetLastError();
     }
-    // blocks of up to 2 048 non-zeros (32 coordinates of 50 on average, with room): the small variant, four CTAs per SM
-    const double avg_block = 32.0 * (double)g.nnz / (double)g.n_coord;
     cudaError_t e;
-    if (avg_block * 1.25 <= 2048.0) {
-        const unsigned grid = stream == g.stream || nb < free_sms * 4 ? nb : free_sms * 4;
-        e = launch_prepare<LOSS, 2048, 2048, 256>(g, P, grid, stream);
+    if (small_prepare(g)) {
+        const unsigned grid = stream == g.stream || nb < free_sms * 3 ? nb : free_sms * 3;
+        e = launch_prepare<LOSS, kPreSmallNz, 2048, 256>(P, grid, stream);
     } else {
-        const unsigned grid = stream == g.stream || nb < free_sms * 2 ? nb : free_sms * 2;
-        e = launch_prepare<LOSS, kMaxNz, kHT, kPreThreadsS>(g, P, grid, stream);
+        const unsigned grid = stream == g.stream || nb < free_sms ? nb : free_sms;
+        e = launch_prepare<LOSS, 4096, 4096, 512>(P, grid, stream);
     }
 #ifdef CHICLE_LA_TIMING
     if (e == cudaSuccess) {
         unsigned long long t[8] = {0};
         (void)cudaStreamSynchronize(stream);
-        (void)cudaMemcpy(t, P.cursor + 16, sizeof(t), cudaMemcpyDeviceToHost);
-        (void)cudaMemset(P.cursor + 16, 0, sizeof(t));
-        fprintf(stderr, "lookahead prepare, cycles per CTA: headers %.0f insert %.0f count %.0f place %.0f number %.0f entries %.0f gram %.0f write %.0f\n",
-                t[0] / (double)nb, t[1] / (double)nb, t[2] / (double)nb, t[3] / (double)nb, t[4] / (double)nb, t[5] / (double)nb,
-                t[6] / (double)nb, t[7] / (double)nb);
+        (void)cudaMemcpy(t, P.timing + 16, sizeof(t), cudaMemcpyDeviceToHost);
+        (void)cudaMemset(P.timing + 16, 0, sizeof(t));
+        const double n = (double)nb;
+        fprintf(stderr, "lookahead prepare, cycles per block: headers %.0f, load + insert %.0f, count %.0f, place %.0f, number %.0f, "
+                "entries %.0f, gram %.0f, cross + write %.0f\n", t[0] / n, t[1] / n, t[2] / n, t[3] / n, t[4] / n, t[5] / n, t[6] / n, t[7] / n);
     }
 #endif
     return e;
 }
 
-// The chain kernel over the blocks that a prepare launch with the same parameters made (on the handle's stream).
 template <int LOSS> cudaError_t launch_chain_on(Glm &g, const LookParams &P)
 {
-    if (g.fmt == CHICLE_FMT_DENSE_ROWMAJOR) return launch_chain<LOSS, true, kCapL, 4, 4>(g, P);
-    if (g.hot_variant) return launch_chain<LOSS, false, kHotSkew, kTmax, 2>(g, P);
-    return launch_chain<LOSS, false, 4, kTmax, 4>(g, P);
+    if (g.fmt == CHICLE_FMT_DENSE_ROWMAJOR) return launch_chain<LOSS, true>(g, P);
+    return launch_chain<LOSS, false>(g, P);
 }
 
-// A round's launches. One slice: prepare, then chain. Several slices (consecutive pieces of every partition's walk):
-// the first slice's prepare on the handle's stream; the later slices' prepares on the side stream, behind the first
-// one, so that they fill the SMs the chain kernels leave idle; every chain launch waits for its slice's prepare.
-template <int LOSS> cudaError_t launch_slices(Glm &g, const LookParams *P, int n_slices)
+// A round's launches, slice after slice (consecutive pieces of every partition's walk). The first slice's prepare
+// kernel runs on the handle's stream; the later ones on the side stream, where they fill the SMs the chain kernels
+// leave idle; every chain launch waits for its slice's prepare kernel. The records of slice s lie in region s mod R
+// of the record buffer, so the prepare kernel of slice s also waits for the chain launch of slice s - R.
+template <int LOSS> cudaError_t launch_slices(Glm &g, std::vector<LookParams> &P)
 {
-    cudaError_t e = launch_prepare_on<LOSS>(g, P[0], g.stream);
+    const int S = (int)P.size(), R = g.la_regions;
+    cudaError_t e = cudaMemsetAsync(g.la_cursor, 0, 4 * sizeof(unsigned long long), g.stream);
+    if (e != cudaSuccess) return e;
+    e = launch_prepare_on<LOSS>(g, P[0], g.stream);
     if (e != cudaSuccess) return e;
     if (g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
-    if (n_slices > 1) {
-        e = cudaEventRecord(g.la_ev[0], g.stream);
+    if (S > 1) {
+        e = cudaEventRecord(g.la_ev_prep[0], g.stream);
         if (e != cudaSuccess) return e;
     }
     e = launch_chain_on<LOSS>(g, P[0]); // enqueued before the side stream's work: it takes its SMs first
-    if (e != cudaSuccess) return e;
-    if (n_slices > 1) {
-        e = cudaStreamWaitEvent(g.la_stream, g.la_ev[0], 0);
-        for (int s = 1; s < n_slices && e == cudaSuccess; ++s) {
-            e = launch_prepare_on<LOSS>(g, P[s], g.la_stream);
-            if (e == cudaSuccess) e = cudaEventRecord(g.la_ev[s], g.la_stream);
+    if (e != cudaSuccess || S == 1) return e;
+    e = cudaEventRecord(g.la_ev_done[0], g.stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(g.la_stream, g.la_ev_prep[0], 0);
+    auto prepare_side = [&](int s) -> cudaError_t {
+        cudaError_t e2 = cudaMemsetAsync(g.la_cursor + (s % R), 0, sizeof(unsigned long long), g.la_stream);
+        if (e2 == cudaSuccess) e2 = launch_prepare_on<LOSS>(g, P[s], g.la_stream);
+        if (e2 == cudaSuccess) e2 = cudaEventRecord(g.la_ev_prep[s], g.la_stream);
+        return e2;
+    };
+    for (int s = 1; s < R && s < S && e == cudaSuccess; ++s) e = prepare_side(s);
+    for (int s = 1; s < S && e == cudaSuccess; ++s) {
+        if (s + R - 1 < S) { // its region is free once the chain launch of slice s - 1 is done
+            e = cudaStreamWaitEvent(g.la_stream, g.la_ev_done[s - 1], 0);
+            if (e == cudaSuccess) e = prepare_side(s + R - 1);
+            if (e != cudaSuccess) break;
         }
-        for (int s = 1; s < n_slices && e == cudaSuccess; ++s) {
-            e = cudaStreamWaitEvent(g.stream, g.la_ev[s], 0);
-            if (e == cudaSuccess) e = launch_chain_on<LOSS>(g, P[s]);
-        }
+        e = cudaStreamWaitEvent(g.stream, g.la_ev_prep[s], 0);
+        if (e == cudaSuccess) e = launch_chain_on<LOSS>(g, P[s]);
+        if (e == cudaSuccess && s + 1 < S) e = cudaEventRecord(g.la_ev_done[s], g.stream);
     }
     return e;
 }
@@ -1097,110 +1722,188 @@ template <int LOSS> cudaError_t launch_slices(Glm &g, const LookParams *P, int n
 } // namespace
 
 int lookahead_max_dense_dim() { return kCapL; }
+int lookahead_max_slices() { return 64; }
+int64_t lookahead_max_dim() { return (int64_t)1 << kIdBits; }
 
-// A round of many blocks is cut into this many slices at most (see launch_slices).
-constexpr int kMaxSlices = 3;
-int lookahead_max_slices() { return kMaxSlices; }
-
-// Bytes of the record buffer and of the block directory that a problem of this shape needs (every block's record at
-// its largest: a head, and 16 bytes per non-zero for the row-wise and the transposed copy; every slice may end in a
-// ragged block per partition).
-void lookahead_workspace(int64_t n_coord, int64_t nnz, int32_t K, bool dense, int64_t dim, size_t *rec_bytes, size_t *dir_bytes)
+// Sizes the look-ahead solver for a partition into K: CTAs per cluster, what stays in shared memory, and the record
+// buffer: `regions` regions that each hold one slice of a round (the recurrence records of its blocks, then a pool
+// for the workers' records).
+void lookahead_plan(Glm &g, int32_t K)
 {
-    const size_t max_blocks = (size_t)(n_coord / kLB + (int64_t)kMaxSlices * (K + 1));
-    *dir_bytes = max_blocks * sizeof(BlkDir);
-    *rec_bytes = max_blocks * (sizeof(BlkHead) + 32) + (dense ? (size_t)n_coord * (size_t)dim * 4 : (size_t)nnz * 16) + 256;
+    const bool dense = g.fmt == CHICLE_FMT_DENSE_ROWMAJOR;
+    int logC = 0;
+    if (!dense && g.hot_variant) {
+        // a cluster per partition, on at most half of the SMs: the prepare kernels need the rest
+        while (logC < 3 && ((int64_t)K << (logC + 1)) * 2 <= g.sm_count) ++logC;
+        const char *env = getenv("CHICLE_LA_CLUSTER");
+        if (env && env[0] >= '1' && env[0] <= '8' && env[1] == 0) {
+            const int want = env[0] - '0';
+            logC = want >= 8 ? 3 : (want >= 4 ? 2 : (want >= 2 ? 1 : 0));
+            while (logC > 0 && ((int64_t)K << logC) > g.sm_count) --logC;
+        }
+    }
+    g.la_logC = logC;
+    const size_t budget = (size_t)(g.max_smem_optin > 0 ? g.max_smem_optin : 227 * 1024);
+    if (dense) {
+        g.la_nzcap = 0;
+        g.la_hotc = (int32_t)g.dim;
+    } else if (!g.hot_variant) {
+        g.la_nzcap = 3072;
+        g.la_hotc = 0;
+    } else {
+        g.la_nzcap = logC == 0 ? 2048 : (logC == 1 ? 1536 : 1024);
+        const ChainLayout L0 = chain_layout(g.la_nzcap, 0, false, (int)g.dim);
+        int64_t hotc = ((int64_t)budget - (int64_t)L0.total - 64) / 4;
+        hotc = hotc < 0 ? 0 : (hotc / 32) * 32;
+        const int64_t need = (g.dim + ((int64_t)1 << logC) - 1) >> logC; // per CTA for the whole model
+        g.la_hotc = (int32_t)(hotc < need ? hotc : (need + 31) / 32 * 32);
+    }
+    g.la_smem = chain_layout(g.la_nzcap, g.la_hotc, dense, (int)g.dim).total;
+
+    // slices: at most a sixteenth of the walk, but at least 256 blocks per partition; three regions
+    const int64_t n = g.n_coord;
+    const int64_t max_nk = (n + K - 1) / K + 1;
+    const int64_t max_nb = (max_nk + kLB - 1) / kLB;
+    int64_t per_part = (max_nb + 15) / 16;
+    per_part = per_part < 256 ? 256 : per_part;
+    per_part = per_part > max_nb ? max_nb : per_part;
+    const bool whole = per_part >= max_nb; // a round is one slice
+    // (partitions of unequal sizes: the largest may hold almost everything; a region then holds what a sixteenth of
+    // the whole walk needs, and the launch cuts finer if a slice does not fit)
+    int64_t region_blocks = whole ? n / kLB + K + 1 : per_part * K + K;
+    if (region_blocks > n / kLB + K + 1) region_blocks = n / kLB + K + 1;
+    g.la_region_blocks = region_blocks;
+    g.la_regions = whole ? 1 : 3;
+    {
+        const char *env = getenv("CHICLE_LA_SLICES"); // forced slicing (tests): the ring as large problems have it
+        if (env && atoi(env) > 1) g.la_regions = 3;
+    }
+    const double frac = whole ? 1.0 : (double)region_blocks / (double)(n / kLB + 1);
+    const size_t C = (size_t)1 << logC;
+    size_t pool;
+    if (dense) pool = (size_t)region_blocks * sub_bytes(kLB * (int)g.dim, 0, true);
+    else {
+        const double all = 14.0 * (double)g.nnz;
+        double part = whole ? all : 1.2 * frac * all + (double)(1 << 20);
+        if (part > all) part = all;
+        pool = (size_t)part + (size_t)region_blocks * C * 128 + 4096;
+    }
+    const size_t heads = ((size_t)region_blocks * sizeof(ChainHead) + 255) & ~(size_t)255;
+    g.la_pool_off = heads;
+    g.la_region_bytes = (heads + pool + 255) & ~(size_t)255;
+    g.la_dir_bytes = (size_t)g.la_regions * (size_t)region_blocks * C * sizeof(BlkDir);
 }
 
 cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
 {
     const int32_t K = g.K;
     std::vector<int64_t> steps((size_t)K), nb((size_t)K);
-    int64_t total = 0, min_nb = (int64_t)1 << 62;
+    int64_t total = 0, max_nb = 0;
     for (int32_t k = 0; k < K; ++k) {
         const int64_t nk = g.h_part_off[k + 1] - g.h_part_off[k];
-        steps[(size_t)k] = g.round_steps ? g.round_steps[k] : (S.H == 0 ? nk : S.H);
+        steps[(size_t)k] = g.round_steps ? g.round_steps[k] : (S.H == 0 ? nk : (nk > 0 ? S.H : 0));
         nb[(size_t)k] = (steps[(size_t)k] + kLB - 1) / kLB;
         total += nb[(size_t)k];
-        if (nb[(size_t)k] > 0 && nb[(size_t)k] < min_nb) min_nb = nb[(size_t)k];
+        if (nb[(size_t)k] > max_nb) max_nb = nb[(size_t)k];
     }
     if (total <= 0 || total > 0x7fffffff) return cudaErrorInvalidConfiguration;
-    // Long walks are cut into slices so that all but the first slice's prepare work runs beside the chain kernels
-    // (which occupy K SMs only; with more than half of the SMs taken by chains the prepare kernels would hold the
-    // chains up instead: such rounds stay in one piece). CHICLE_LA_SLICES=1 keeps every round in one piece (to time the prepare kernel alone),
-    // CHICLE_LA_SLICES=3 cuts short walks too (to test the slicing on small problems).
-    const bool can_slice = g.la_stream && g.la_slice && min_nb >= 8; // every partition has blocks in every slice
-    int n_slices = (can_slice && total >= 4096 && min_nb >= 64 && 2 * K <= g.sm_count) ? kMaxSlices : 1;
+    // Slices: fractions 0 = F_0 < F_1 < ... < F_S = 1 of every partition's walk. The first slice is small (its
+    // prepare kernel is the one nothing hides), the next ones double, up to a sixteenth of the walk or 256 blocks of
+    // the longest partition, whichever is more; a slice must fit a region of the record buffer.
+    // CHICLE_LA_SLICES=1 keeps every round in one piece (to time the prepare kernel alone), CHICLE_LA_SLICES=n cuts
+    // into n equal slices whatever the length (to test the slicing on small problems).
+    const int max_slices = lookahead_max_slices();
+    std::vector<double> F;
     const char *env = getenv("CHICLE_LA_SLICES");
-    if (env && env[0] == '1' && env[1] == 0) n_slices = 1;
-    if (env && env[0] == '3' && env[1] == 0 && can_slice) n_slices = kMaxSlices;
-
-    LookParams P[kMaxSlices];
-    for (int s = 0; s < kMaxSlices; ++s) {
-        P[s] = LookParams{};
-        P[s].S = S;
-        P[s].rec = static_cast<unsigned char *>(g.la_rec);
-        P[s].cursor = g.la_cursor;
-        P[s].rec_cap = g.la_rec_bytes;
-        P[s].K = K;
-    }
-    cudaError_t e = cudaMemsetAsync(g.la_cursor, 0, sizeof(unsigned long long), g.stream);
-    if (e != cudaSuccess) return e;
-    if (n_slices == 1) {
-        P[0].dir = static_cast<BlkDir *>(g.la_dir);
-        P[0].blk_base = g.la_blk_base;
-        P[0].n_blocks = total;
-        k_block_bases<<<1, 32, 0, g.stream>>>(P[0].S, K, g.la_blk_base);
+    const int forced = env ? atoi(env) : 0;
+    auto build = [&](double first, double cap) {
+        F.assign(1, 0.0);
+        double at = 0.0, len = first;
+        while (at < 1.0 && (int)F.size() < max_slices) {
+            at += len;
+            F.push_back(at < 1.0 ? at : 1.0);
+            len = len * 2.0 < cap ? len * 2.0 : cap;
+        }
+        F.back() = 1.0;
+    };
+    double cap = 1.0;
+    if (forced >= 1 && (forced == 1 || g.la_stream)) {
+        const int n = forced > max_slices ? max_slices : forced;
+        F.assign(1, 0.0);
+        for (int s = 1; s <= n; ++s) F.push_back((double)s / n);
+    } else if (!g.la_stream || g.la_regions == 1 || max_nb < 512) {
+        F = {0.0, 1.0};
     } else {
-        // Slice s of partition k: blocks cut[s] .. cut[s + 1] of its walk. The prepare kernel of slice s + 1 should
-        // be done when the chain launch of slice s is, so the slices grow by a factor a = 0.8 / rho, where rho is the
-        // prepare time of a piece of the walk on the SMs the chains leave over its chain time: about
-        // c K / (SMs - K) with c = SM-time of the prepare kernel per step over the chain's time per step, 1.2 to
-        // 1.9 measured on the sparse configurations (2 assumed), 0.18 on short dense rows (0.25 assumed). The first
-        // slice's prepare kernel is the part that stays exposed: 1 / (1 + a + a^2) of the walk.
-        const double c_ratio = g.fmt == CHICLE_FMT_DENSE_ROWMAJOR ? 0.25 : 2.0;
-        const double rho = c_ratio * (double)K / (double)(g.sm_count > K ? g.sm_count - K : 1);
-        const double a = 0.8 / rho;
-        double f1 = 1.0 / (1.0 + a + a * a);
-        f1 = f1 < 1.0 / 64 ? 1.0 / 64 : (f1 > 0.5 ? 0.5 : f1);
-        const double f2 = a * f1;
-        std::vector<int64_t> h((size_t)kMaxSlices * 2 * (size_t)K);
-        int64_t blocks[kMaxSlices] = {0, 0, 0};
+        cap = 1.0 / 16;
+        if (cap * (double)max_nb < 256.0) cap = 256.0 / (double)max_nb;
+        build(cap / 8, cap);
+    }
+    std::vector<int64_t> h;
+    std::vector<int64_t> blocks;
+    for (int attempt = 0; attempt < 24; ++attempt) {
+        const int Sn = (int)F.size() - 1;
+        h.assign((size_t)Sn * 2 * (size_t)K, 0);
+        blocks.assign((size_t)Sn, 0);
+        int64_t worst = 0;
         for (int32_t k = 0; k < K; ++k) {
-            const int64_t nbk = nb[(size_t)k]; // 0, or at least 8
-            int64_t c1 = (int64_t)((double)nbk * f1), c2 = (int64_t)((double)nbk * (f1 + f2));
-            c1 = c1 < 1 ? 1 : c1;
-            c2 = c2 < c1 + 1 ? c1 + 1 : c2;
-            c2 = c2 > nbk - 1 ? nbk - 1 : c2;
-            const int64_t cut[kMaxSlices + 1] = {0, nbk ? c1 : 0, nbk ? c2 : 0, nbk};
-            for (int s = 0; s < kMaxSlices; ++s) {
-                const int64_t first = cut[s] * kLB;
-                const int64_t last = s + 1 == kMaxSlices ? steps[(size_t)k] : cut[s + 1] * kLB;
+            const int64_t nbk = nb[(size_t)k];
+            int64_t prev = 0;
+            for (int s = 0; s < Sn; ++s) {
+                int64_t cut = s + 1 == Sn ? nbk : (int64_t)((double)nbk * F[(size_t)s + 1]);
+                cut = cut < prev ? prev : (cut > nbk ? nbk : cut);
+                const int64_t first = prev * kLB;
+                const int64_t last = s + 1 == Sn ? steps[(size_t)k] : cut * kLB;
                 h[((size_t)s * 2) * (size_t)K + (size_t)k] = last - first;
                 h[((size_t)s * 2 + 1) * (size_t)K + (size_t)k] = first;
-                blocks[s] += (last - first + kLB - 1) / kLB;
+                blocks[(size_t)s] += (last - first + kLB - 1) / kLB;
+                prev = cut;
             }
         }
-        // a pageable source: the runtime has taken its copy of these words when the call returns
-        e = cudaMemcpyAsync(g.la_slice, h.data(), h.size() * sizeof(int64_t), cudaMemcpyHostToDevice, g.stream);
-        if (e != cudaSuccess) return e;
-        int64_t dir_off = 0;
-        for (int s = 0; s < kMaxSlices; ++s) {
-            P[s].S.H = 0;
-            P[s].S.steps_k = g.la_slice + ((size_t)s * 2) * (size_t)K;
-            P[s].S.first_k = g.la_slice + ((size_t)s * 2 + 1) * (size_t)K;
-            P[s].dir = static_cast<BlkDir *>(g.la_dir) + dir_off;
-            int64_t *bases = g.la_blk_base + (size_t)s * ((size_t)K + 1);
-            P[s].blk_base = bases;
-            P[s].n_blocks = blocks[s];
-            dir_off += blocks[s];
-            k_block_bases<<<1, 32, 0, g.stream>>>(P[s].S, K, bases);
-        }
+        for (int s = 0; s < Sn; ++s) worst = blocks[(size_t)s] > worst ? blocks[(size_t)s] : worst;
+        if (worst <= g.la_region_blocks) break;
+        // finer: equal slices, twice as many as would just fit
+        int n = (int)((total + g.la_region_blocks - 1) / g.la_region_blocks) * (attempt + 2);
+        if (n > max_slices) n = max_slices;
+        if (!g.la_stream || g.la_regions < 2 || attempt == 23) return cudaErrorInvalidConfiguration;
+        F.assign(1, 0.0);
+        for (int s = 1; s <= n; ++s) F.push_back((double)s / n);
     }
+    const int Sn = (int)F.size() - 1;
+    // a pageable source: the runtime has taken its copy of these words when the call returns
+    cudaError_t e = cudaMemcpyAsync(g.la_slice, h.data(), h.size() * sizeof(int64_t), cudaMemcpyHostToDevice, g.stream);
+    if (e != cudaSuccess) return e;
+    k_block_bases_slices<<<Sn, 32, 0, g.stream>>>(g.la_slice, K, g.la_blk_base);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const char *drop = getenv("CHICLE_TEST_DROP_RECORD"); // test aid: leave one block's records unpublished
+    const size_t C = (size_t)1 << g.la_logC;
+    std::vector<LookParams> P((size_t)Sn);
+    for (int s = 0; s < Sn; ++s) {
+        const int r = s % g.la_regions;
+        LookParams &p = P[(size_t)s];
+        p = LookParams{};
+        p.S = S;
+        p.S.H = 0;
+        p.S.steps_k = g.la_slice + ((size_t)s * 2) * (size_t)K;
+        p.S.first_k = g.la_slice + ((size_t)s * 2 + 1) * (size_t)K;
+        p.rec = static_cast<unsigned char *>(g.la_rec) + (size_t)r * g.la_region_bytes;
+        p.dirS = static_cast<BlkDir *>(g.la_dir) + (size_t)r * (size_t)g.la_region_blocks * C;
+        p.cursor = g.la_cursor + r;
+        p.timing = g.la_cursor + 8;
+        p.pool_off = g.la_pool_off;
+        p.pool_cap = g.la_region_bytes - g.la_pool_off;
+        p.blk_base = g.la_blk_base + (size_t)s * ((size_t)K + 1);
+        p.K = K;
+        p.logC = g.la_logC;
+        p.nzcap = g.la_nzcap;
+        p.hotc = g.la_hotc;
+        p.n_blocks = blocks[(size_t)s];
+        p.drop_block = (drop && s == 0) ? atoll(drop) : -1;
+    }
+    g.la_last_slices = Sn;
     switch (g.loss) {
-    case CHICLE_LOSS_HINGE_DUAL: return launch_slices<CHICLE_LOSS_HINGE_DUAL>(g, P, n_slices);
-    case CHICLE_LOSS_LOGISTIC_DUAL: return launch_slices<CHICLE_LOSS_LOGISTIC_DUAL>(g, P, n_slices);
-    default: return launch_slices<CHICLE_LOSS_RIDGE_PRIMAL>(g, P, n_slices);
+    case CHICLE_LOSS_HINGE_DUAL: return launch_slices<CHICLE_LOSS_HINGE_DUAL>(g, P);
+    case CHICLE_LOSS_LOGISTIC_DUAL: return launch_slices<CHICLE_LOSS_LOGISTIC_DUAL>(g, P);
+    default: return launch_slices<CHICLE_LOSS_RIDGE_PRIMAL>(g, P);
     }
 }
 
