@@ -91,6 +91,10 @@ typedef struct {
                              the prepare kernel of the whole round, or of its first slice when a long round is cut
                              into slices whose prepare kernels run beside the chain kernels; when H spans several
                              local epochs: the first epoch's; else 0 */
+    int32_t solver_slices;   /* look-ahead solver: slices the round's walk was cut into (last local epoch); else 0   */
+    int32_t cluster_ctas;    /* look-ahead solver: CTAs per partition (thread-block cluster size); else 1            */
+    int32_t solver_launches; /* kernels the local solvers launched in this round (block tables, prepare, chain)      */
+    int32_t order_launches;  /* kernels launched for this round's visiting orders                                    */
 } chicle_round_stats_t;
 
 /* Create a training problem (Sec. 2.2, Sec. 5.1: a GLM trained by CoCoA with a local SCD solver; Sec. 4.4:
@@ -232,7 +236,12 @@ chicle_status_t chicle_get_info(const chicle_glm_t *h, int64_t *round, int32_t *
  *   host_errbuf           optional host buffer of errbuf_len bytes that receives the error text (no handle exists to
  *                         keep it). The caller owns both output arrays and the buffer.
  * The first call on a device looks up the device address of the workspace (cudaGetSymbolAddress) and remembers it;
- * make that first call outside any stream capture. All calls on a device share the one workspace, and it keeps
+ * make that first call outside any stream capture. That first call is also the one exception to "allocates
+ * nothing": the CUDA runtime loads kernels and static device arrays lazily, so the lookup and the first launch of
+ * each kernel may make the driver set device memory aside for the library's image. Callers with a frozen memory
+ * budget make one call at start-up, before the region in which nothing may be allocated; every later call on that
+ * device leaves the free device memory as it found it. The call makes `device` the current device of the calling
+ * thread and leaves it so. All calls on a device share the one workspace, and it keeps
  * whatever the previous call left in it; nothing in it needs clearing because every pass overwrites what it then
  * reads. Two calls whose kernels overlap on the same GPU (different streams, or different host threads) race on it:
  * serialise them. Results are bit-identical to chicle_partition's. */

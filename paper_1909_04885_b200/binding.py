@@ -15,7 +15,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("CHICLE_LIB_PATH") or os.path.join(_HERE, "libchicle.so")
 
-OK = 0
+OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED, ERR_NUMERIC, ERR_TIMEOUT = range(8)
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_STATE", 3: "OOM", 4: "CUDA", 5: "UNSUPPORTED", 6: "NUMERIC", 7: "TIMEOUT"}
 LOSS = {"hinge": 0, "logistic": 1, "ridge": 2}
 FMT = {"dense": 0, "csr": 1, "csc": 2}
@@ -49,7 +49,9 @@ class Allocator(C.Structure):
 
 class RoundStats(C.Structure):
     _fields_ = [("ms_permutation", C.c_float), ("ms_local", C.c_float), ("ms_reduce", C.c_float), ("ms_total", C.c_float),
-                ("steps", C.c_int64), ("solver_variant", C.c_int32), ("ms_prepare", C.c_float)]
+                ("steps", C.c_int64), ("solver_variant", C.c_int32), ("ms_prepare", C.c_float),
+                ("solver_slices", C.c_int32), ("cluster_ctas", C.c_int32), ("solver_launches", C.c_int32),
+                ("order_launches", C.c_int32)]
 
 
 _lib = None
@@ -131,11 +133,14 @@ class _TorchAllocator:
         self._torch = torch
         self._device = torch.device("cuda", device)
         self._live = {}
+        self.fail = False   # True: every request is refused (the callback returns NULL), to exercise the library's OOM paths
         self._alloc_cb = ALLOC_FN(self._alloc)
         self._free_cb = FREE_FN(self._free)
         self.struct = Allocator(self._alloc_cb, self._free_cb, None)
 
     def _alloc(self, _ctx, nbytes):
+        if self.fail:
+            return None
         try:
             t = self._torch.empty(int(nbytes), dtype=self._torch.uint8, device=self._device)
         except Exception:
@@ -257,8 +262,16 @@ class Glm:
         if stats:
             return {"ms_permutation": rs.ms_permutation, "ms_local": rs.ms_local, "ms_reduce": rs.ms_reduce,
                     "ms_total": rs.ms_total, "steps": rs.steps, "solver_variant": rs.solver_variant,
-                    "ms_prepare": rs.ms_prepare}
+                    "ms_prepare": rs.ms_prepare, "solver_slices": rs.solver_slices, "cluster_ctas": rs.cluster_ctas,
+                    "solver_launches": rs.solver_launches, "order_launches": rs.order_launches}
         return None
+
+    def fail_allocations(self, on: bool):
+        """Makes the allocator callback that the library was given refuse every request (return NULL) from now on, or
+        serve them again: a way to see the library's out-of-memory behaviour without exhausting the device."""
+        if self._alloc is None:
+            raise RuntimeError("this handle allocates with cudaMalloc, not through a callback")
+        self._alloc.fail = bool(on)
 
     def duality_gap(self):
         g, p, d = C.c_double(), C.c_double(), C.c_double()

@@ -494,6 +494,7 @@ static chicle_status_t round_impl(chicle_glm_t *h, int64_t H, const int64_t *hos
     if (stats) (void)cudaEventRecord(h->ev[1], s);
     int variant = 0;
     h->time_prepare = stats != nullptr;
+    h->solver_launches = 0;
     if (host_steps) {
         // a pageable source: the runtime has taken its copy of the K words when the call returns
         e = cudaMemcpyAsync(h->d_steps, host_steps, (size_t)h->K * sizeof(int64_t), cudaMemcpyHostToDevice, s);
@@ -526,6 +527,10 @@ static chicle_status_t round_impl(chicle_glm_t *h, int64_t H, const int64_t *hos
         r.steps = steps;
         r.solver_variant = variant;
         if (variant >= 4) (void)cudaEventElapsedTime(&r.ms_prepare, h->ev[1], h->ev[4]);
+        r.solver_slices = variant >= 4 ? h->la_last_slices : 0;
+        r.cluster_ctas = variant == 4 ? (1 << h->la_logC) : 1;
+        r.solver_launches = steps > 0 ? (h->solver_launches > 0 ? h->solver_launches : 1) : 0;
+        r.order_launches = (int32_t)(epochs * (22 + 5 * (h->K <= 256 ? 1 : 2)));
         *stats = r;
     }
     return CHICLE_OK;

@@ -110,6 +110,7 @@ struct Glm {
     int32_t la_nzcap = 0, la_hotc = 0; // non-zeros per worker record; entry ids per CTA kept in shared memory
     size_t la_smem = 0;              // dynamic shared memory of the chain kernel
     int la_last_slices = 0;          // slices of the last round
+    int solver_launches = 0;         // kernels the local solvers launched in the round being enqueued
     int64_t *la_blk_base = nullptr;  // per slice K+1: first block of each partition in the slice's numbering of the blocks
     int64_t *la_slice = nullptr;     // per slice 2K: every partition's step count and first step in that slice
     cudaStream_t la_stream = nullptr; // side stream (lowest priority) for the later slices' prepare kernels

@@ -374,19 +374,75 @@ def test_gap_tile_that_does_not_fit_a_stage_is_read_in_place():
     run_parity(wl)
 
 
-def test_lookahead_runs_are_bit_reproducible():
-    w = datagen.make("hinge_csr", 100)
+@pytest.mark.parametrize("name,scale,slices", [("hinge_csr", 100, None), ("ridge_csc", 100, None), ("hinge_dense", 1, None),
+                                               ("logistic_dense", 100, None), ("hinge_hashed", 1000, "3")])
+def test_lookahead_runs_are_bit_reproducible(name, scale, slices, monkeypatch):
+    # the skewed variant (part of the model in shared memory, split over a cluster), the flat one (every id goes through
+    # reductions on the update rows in global memory), the dense one, and a round cut into slices
+    if slices:
+        monkeypatch.setenv("CHICLE_LA_SLICES", slices)
+    w = datagen.make(name, scale)
+    ph = w.phases[0]
     res = []
     for _ in range(2):
         glm = binding.from_workload(w)
         try:
-            glm.partition(16, 0)
+            glm.partition(ph.K, ph.seed)
             for _ in range(3):
-                glm.cocoa_round(0, 16.0)
-            res.append((glm.get_alpha().copy(), glm.get_v().copy()))
+                glm.cocoa_round(0, ph.sigma_prime)
+            res.append((glm.get_alpha().copy(), glm.get_v().copy(), glm.duality_gap()["gap"]))
         finally:
             glm.close()
-    assert np.array_equal(res[0][0], res[1][0]) and np.array_equal(res[0][1], res[1][1])
+    assert np.array_equal(res[0][0], res[1][0]) and np.array_equal(res[0][1], res[1][1]) and res[0][2] == res[1][2]
+
+
+def test_a_missing_record_ends_in_a_timeout_status_and_the_handle_stays_usable(monkeypatch):
+    # Failure detection without a fault: one block's records are left unpublished (a host-side test aid), so the chain
+    # kernel finds nothing to copy, sets the status word with no copy in flight, every wait in the cluster runs out
+    # within its bound, all roles return, and the call reports the timeout. The handle then takes a new partition
+    # and runs on.
+    w = datagen.make("hinge_csr", 200)
+    ph = w.phases[0]
+    orc, glm = make_pair(w)
+    try:
+        glm.partition(ph.K, ph.seed)
+        monkeypatch.setenv("CHICLE_TEST_DROP_RECORD", "3")
+        with pytest.raises(binding.ChicleError) as e:
+            glm.cocoa_round(0, ph.sigma_prime)
+            glm.duality_gap()     # (the status word is read by the next synchronising call)
+        assert e.value.status == binding.ERR_TIMEOUT
+        monkeypatch.delenv("CHICLE_TEST_DROP_RECORD")
+        # the state is whatever the aborted round left: start again from the oracle's
+        glm.set_state(orc.state.astype(np.float32), orc.v.astype(np.float32), 0)
+        orc.partition(ph.K, ph.seed)
+        glm.partition(ph.K, ph.seed)
+        orc.cocoa_round(0, ph.sigma_prime)
+        glm.cocoa_round(0, ph.sigma_prime)
+        assert rel_l2(glm.get_alpha(), orc.state) <= 1e-4 and rel_l2(glm.get_v(), orc.v) <= 1e-4
+    finally:
+        glm.close()
+
+
+def test_allocator_that_returns_null_gives_oom(monkeypatch):
+    # host-side fault injection: the allocator callback starts returning NULL
+    w = tiny_csr(300, 40, seed=3, K=3)
+    glm = binding.from_workload(w)
+    try:
+        glm.partition(3, 0)
+        glm.cocoa_round(0, 3.0)
+        glm.fail_allocations(True)
+        with pytest.raises(binding.ChicleError) as e:
+            glm.partition(5, 1)          # needs a new K x d update workspace
+        assert e.value.status == binding.ERR_OOM
+        glm.fail_allocations(False)
+        with pytest.raises(binding.ChicleError) as e:
+            glm.cocoa_round(0, 3.0)      # documented: the failed call released the old workspace, the handle has no partition
+        assert e.value.status == binding.ERR_BAD_STATE
+        glm.partition(5, 1)
+        glm.cocoa_round(0, 5.0)
+        assert glm.duality_gap()["gap"] >= 0
+    finally:
+        glm.close()
 
 
 def test_round_stats():
