@@ -107,6 +107,8 @@ struct Glm {
     int64_t la_region_blocks = 0;    // blocks a region has records for
     int la_regions = 0;
     int la_logC = 0;                 // log2 of the CTAs per partition (thread-block cluster)
+    int la_depth = 2;                // blocks the dot products are taken ahead of the recurrence (2: with cross Gram matrices)
+    bool la_overlap = true;          // prepare kernels beside the chain kernels (side stream) or alternating with them
     int32_t la_nzcap = 0, la_hotc = 0; // non-zeros per worker record; entry ids per CTA kept in shared memory
     size_t la_smem = 0;              // dynamic shared memory of the chain kernel
     int la_last_slices = 0;          // slices of the last round

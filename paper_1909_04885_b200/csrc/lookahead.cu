@@ -111,6 +111,8 @@ struct LookParams {
     unsigned long long pool_cap; // bytes of the pool
     const int64_t *blk_base;     // K + 1: the first block of each partition in this launch's numbering of the blocks
     int32_t K, logC;
+    int32_t depth;               // 2: a block's dot products are taken two blocks ahead and corrected with the cross
+                                 // Gram matrix; 1: one block ahead, no cross Gram matrix (the recurrence waits for them)
     int32_t nzcap;               // non-zeros a worker record holds at most
     int32_t hotc;                // entry ids per CTA kept in shared memory
     int64_t n_blocks;
@@ -229,8 +231,6 @@ template <int HT> __device__ __forceinline__ uint32_t home_slot(int32_t id)
 template <int HT> __device__ __forceinline__ uint32_t next_slot(uint32_t p) { return p + 1 < (uint32_t)HT ? p + 1 : kHD; }
 
 // ------------------------------------------------------------------------------------------------ prepare
-constexpr int kScanVals = 1 + kMaxC;
-
 template <int NZ, int HT, int THREADS> struct PreShared {
     int32_t idx[NZ];     // the block's non-zeros, row after row (later: the membership mask of the non-zero's id)
     float val[NZ];
@@ -250,7 +250,7 @@ template <int NZ, int HT, int THREADS> struct PreShared {
     int32_t nnz[kLB];
     int32_t roff[kLB + 1];
     uint16_t rc[kLB + 1][kMaxC]; // non-zeros of coordinate j that fall to CTA c; then where they start in c's record
-    uint32_t warp_tot[THREADS / 32][kScanVals];
+    uint32_t cntTL[kMaxC], cntTL2[kMaxC], cntAll; // per CTA: shared ids (high half) and their list entries (low half); all list entries
     float gsc[kLB], ys[kLB], as[kLB]; // per coordinate: its Gram scale, and what multiplies / enters from the earlier ones
     float gscn[kLB];                  // the next block's coordinates: their Gram scales
     int64_t nrs[kLB];
@@ -277,7 +277,7 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
     const int64_t steps = steps_of(P, k, nk);
     const int cnt = (int)((steps - b * kLB) < kLB ? (steps - b * kLB) : kLB);
     const int64_t left = steps - (b + 1) * kLB; // steps behind this block
-    const int ncnt = left <= 0 ? 0 : (left < kLB ? (int)left : kLB);
+    const int ncnt = (left <= 0 || P.depth < 2) ? 0 : (left < kLB ? (int)left : kLB);
     ChainHead &out = *reinterpret_cast<ChainHead *>(P.rec + (size_t)bid * sizeof(ChainHead));
 #ifdef CHICLE_LA_TIMING
     long long pt0 = clock64(), pt1 = 0;
@@ -347,7 +347,8 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
         (&sh.Dc[0][0])[p] = 0.0f;
         (&sh.Dn[0][0])[p] = 0.0f;
     }
-    if (tid < kMaxC) sh.ncls[tid] = 0;
+    if (tid < kMaxC) { sh.ncls[tid] = 0; sh.cntTL[tid] = 0u; sh.cntTL2[tid] = 0u; }
+    if (tid == 0) sh.cntAll = 0u;
     __syncthreads();
     PRE_T(0);
     const int total = sh.total;
@@ -412,38 +413,14 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
     }
     __syncthreads();
     PRE_T(1);
-    // ---- number the ids: every id's list of values for the Gram passes (soff), and for the ids that more than one
-    //      coordinate has, their number and their list's start inside their CTA's record. Thread t owns slots t,
-    //      t + THREADS, ...; its running counts follow those of the threads before it. v[0]: list entries of all ids;
-    //      v[1 + c]: CTA c's shared ids in the high half, their list entries in the low half.
-    uint32_t v[kScanVals];
-#pragma unroll
-    for (int i = 0; i < kScanVals; ++i) v[i] = 0u;
+    // ---- count the ids that more than one coordinate has, and their list entries, per CTA (shared-memory atomics:
+    //      ids in the high half, list entries in the low half; only the totals are needed before the records' places
+    //      are known)
     if (!slow)
         for (int p = tid; p < HT; p += THREADS) {
             const uint32_t m = sh.mask[p];
-            if (m == 0u) continue;
-            const uint32_t pc = (uint32_t)__popc(m);
-            v[0] += pc;
-            if (m & (m - 1u)) {
-                const int c = sh.key[p] & (C - 1);
-#pragma unroll
-                for (int i = 0; i < kMaxC; ++i)
-                    if (i == c) v[1 + i] += (1u << 16) + pc;
-            }
+            if (m & (m - 1u)) atomicAdd(&sh.cntTL[sh.key[p] & (C - 1)], (1u << 16) + (uint32_t)__popc(m));
         }
-    uint32_t run[kScanVals];
-#pragma unroll
-    for (int i = 0; i < kScanVals; ++i) {
-        uint32_t incl = v[i];
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += t;
-        }
-        if (lane == 31) sh.warp_tot[warp][i] = incl;
-        run[i] = incl - v[i];
-    }
     // where each coordinate's non-zeros start in each CTA's record (warp 0, lane = coordinate)
     if (warp == 0 && !slow) {
 #pragma unroll
@@ -461,15 +438,6 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
     }
     __syncthreads();
     PRE_T(2);
-    uint32_t all[kScanVals];
-#pragma unroll
-    for (int i = 0; i < kScanVals; ++i) {
-        all[i] = 0u;
-        for (int w2 = 0; w2 < NW; ++w2) {
-            if (w2 < warp) run[i] += sh.warp_tot[w2][i];
-            all[i] += sh.warp_tot[w2][i];
-        }
-    }
     // ---- the records' places: the head has its own (one per block); the workers' records come from the pool. A
     //      block that the pool has no room for is walked in place like one that is too long.
     if (tid == 0) {
@@ -477,7 +445,7 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
         uint32_t len[kMaxC];
 #pragma unroll
         for (int c = 0; c < kMaxC; ++c) {
-            len[c] = c < C ? sub_bytes(sh.rc[kLB][c], (int)(all[1 + c] >> 16), false) : 0u;
+            len[c] = c < C ? sub_bytes(sh.rc[kLB][c], (int)(sh.cntTL[c] >> 16), false) : 0u;
             need += len[c];
         }
         unsigned long long at = 0;
@@ -504,7 +472,7 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
                 d.flags = 0u;
                 sh.sub_off[c] = d.offset;
                 sh.sub_len[c] = len[c];
-                sh.subT[c] = (int32_t)(all[1 + c] >> 16);
+                sh.subT[c] = (int32_t)(sh.cntTL[c] >> 16);
                 at += len[c];
             }
             if (bid == P.drop_block) d.bytes = 0u;
@@ -543,16 +511,14 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
     for (int p = tid; p < HT; p += THREADS) {
         const uint32_t m = sh.mask[p];
         if (m == 0u) continue;
+        // (numbered with atomics: the order varies from run to run, which moves records' contents about but changes no
+        // result: every id's own sum is taken in coordinate order, in a shape that depends on the list's length alone)
         const uint32_t pc = (uint32_t)__popc(m);
-        sh.soff[p] = (uint16_t)run[0];
-        run[0] += pc;
+        sh.soff[p] = (uint16_t)atomicAdd(&sh.cntAll, pc);
         if (m & (m - 1u)) {
             const int32_t id = sh.key[p];
             const int c = id & (C - 1);
-            uint32_t r = 0u;
-#pragma unroll
-            for (int i = 0; i < kMaxC; ++i)
-                if (i == c) { r = run[1 + i]; run[1 + i] += (1u << 16) + pc; }
+            const uint32_t r = atomicAdd(&sh.cntTL2[c], (1u << 16) + pc);
             const uint32_t t = r >> 16, o = r & 0xffffu;
             unsigned char *rec = P.rec + sh.sub_off[c];
             const int n_c = sh.rc[kLB][c], T_c = sh.subT[c];
@@ -560,14 +526,13 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
             uint16_t *off_g = reinterpret_cast<uint16_t *>(rec + sizeof(SubHead) + 8u * n_c + 4u * T_c + 2u * n_c);
             ids_g[t] = (uint32_t)id;
             off_g[t] = (uint16_t)o;
-            if ((int)t == T_c - 1) off_g[T_c] = (uint16_t)(o + pc);
             sh.coff[p] = (uint16_t)o;
         }
     }
-    if (tid < C && sh.subT[tid] == 0) { // no shared ids: the list of starts is its end alone
+    if (tid < C) { // the end of the last list
         unsigned char *rec = P.rec + sh.sub_off[tid];
-        const int n_c = sh.rc[kLB][tid];
-        reinterpret_cast<uint16_t *>(rec + sizeof(SubHead) + 8u * n_c + 2u * n_c)[0] = 0;
+        const int n_c = sh.rc[kLB][tid], T_c = sh.subT[tid];
+        reinterpret_cast<uint16_t *>(rec + sizeof(SubHead) + 8u * n_c + 4u * T_c + 2u * n_c)[T_c] = (uint16_t)(sh.cntTL[tid] & 0xffffu);
     }
     __syncthreads();
     PRE_T(4);
@@ -808,7 +773,7 @@ template <int LOSS> __device__ __forceinline__ void prepare_block_dense(const Lo
     const int64_t steps = steps_of(P, k, nk);
     const int cnt = (int)((steps - b * kLB) < kLB ? (steps - b * kLB) : kLB);
     const int64_t left = steps - (b + 1) * kLB;
-    const int ncnt = left <= 0 ? 0 : (left < kLB ? (int)left : kLB);
+    const int ncnt = (left <= 0 || P.depth < 2) ? 0 : (left < kLB ? (int)left : kLB);
     const int dim = (int)P.S.dim;
     ChainHead &out = *reinterpret_cast<ChainHead *>(P.rec + (size_t)bid * sizeof(ChainHead));
     if (tid == 0) {
@@ -1325,15 +1290,22 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
             load_dir(3, d); issue_sub(3, d); sl3 = nb > 3 && (d[3] & 1u) != 0u;
         }
         int64_t fg = 0; // staged blocks whose dot products have been sent
+        bool failed = false; // this warp gave up a wait (voted on at the next barrier)
 #ifdef CHICLE_LA_TIMING
         long long wd = 0, ws = 0, wg = 0, ws1 = 0, wg0 = 0, wg1 = 0, t0 = clock64(), t1 = 0;
 #endif
 
         // Block x's dot products against the model as it is now (this CTA's part), sent to CTA 0.
         auto take_dots = [&](int64_t x) -> bool {
-            bool ok = wt >= 32 || mbar_wait_cluster(smem_u32(&ctl.subfull[x & (kSubSlots - 1)]), (uint32_t)(x >> 2) & 1u, abort_flag, S.status);
-            ok = work_bar_and(ok); // (also: the products of the phase before have been read)
-            if (!ok) return false;
+            // Every warp waits for the record by itself (a barrier costs more than 200 cycles); a warp whose wait runs out
+            // skips the work and says so at the next barrier's vote, so that all warps still meet there.
+            bool ok = mbar_wait_cluster(smem_u32(&ctl.subfull[x & (kSubSlots - 1)]), (uint32_t)(x >> 2) & 1u, abort_flag, S.status);
+            if (DENSE) ok = work_bar_and(ok); // (dense rows: the products of the call before have been read)
+            if (!ok) {
+                failed = true;
+                ++fg;
+                return !DENSE;
+            }
             LA_T(wg0);
             const unsigned char *rec = sub_at(x);
             const SubHead &h = *reinterpret_cast<const SubHead *>(rec);
@@ -1378,10 +1350,24 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                     }
                     float acc = x[0] * (cold[0] ? fmaf(sigma, uu[0], vb[0]) : hv[0]);
                     acc = fmaf(x[1], cold[1] ? fmaf(sigma, uu[1], vb[1]) : hv[1], acc);
-                    for (int e = lo + 16; e < hi; e += 8) {
-                        const uint32_t g = meta[e] & kIdMask;
-                        const float ww = g < hot_total ? W[g >> logC] : fmaf(sigma, __ldcg(Uk + g), S.vbase[g]);
-                        acc = fmaf(val[e], ww, acc);
+                    // (longer coordinates: four at a time, again with all loads first: an id beyond the part of the
+                    // model in shared memory costs a round trip to L2, which the four share)
+                    for (int e0 = lo + 16; e0 < hi; e0 += 32) {
+                        float x4[4], h4[4], u4[4], v4[4];
+                        bool c4[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int e = e0 + 8 * u;
+                            const bool on = e < hi;
+                            x4[u] = on ? val[e] : 0.0f;
+                            const uint32_t g = on ? (meta[e] & kIdMask) : 0u;
+                            c4[u] = on && g >= hot_total;
+                            h4[u] = W[c4[u] ? 0u : (g >> logC)];
+                            u4[u] = ldcg_if(Uk + (c4[u] ? g : 0u), c4[u]);
+                            v4[u] = ldca_if(S.vbase + (c4[u] ? g : 0u), c4[u]);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) acc = fmaf(x4[u], c4[u] ? fmaf(sigma, u4[u], v4[u]) : h4[u], acc);
                     }
                     acc += __shfl_xor_sync(0xffffffffu, acc, 1);
                     acc += __shfl_xor_sync(0xffffffffu, acc, 2);
@@ -1394,23 +1380,27 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
             return true;
         };
 
-        if (!sl0) aborted = !take_dots(0);
-        if (!aborted && nb > 1 && !sl0 && !sl1) aborted = !take_dots(1);
-        LA_T(wg);
-        for (int64_t b = 0; b < nb && !aborted; ++b) {
+        // The loop starts `depth` blocks early: those turns only take the first blocks' dot products (one place in the
+        // code for every phase keeps the loop small: the warps run at the pace instructions can be fetched).
+        const int depth = P.depth;
+        if (depth == 2) { sl2 = sl0; sl3 = sl1; sl0 = false; sl1 = false; } // flags of blocks b .. b + 3 for b = -2
+        else { sl3 = sl2; sl2 = sl1; sl1 = sl0; sl0 = false; }              // ... for b = -1
+#pragma unroll 1
+        for (int64_t b = -depth; b < nb && !aborted; ++b) {
             uint32_t dn[4];
             load_dir(b + kSubSlots, dn);
             const uint32_t par = (uint32_t)(b & 1);
-            if (sl0) {
+            if (b < 0) {
+            } else if (sl0) {
                 // walked in place by CTA 0: every update before it has been applied here (the barrier that ended
                 // the block before); say so, and wait for the walk to end
                 if (wt == 0) mbar_arrive_remote_release(ack_bar);
-                bool ok = wt >= 32 || mbar_wait_cluster(smem_u32(&ctl.dbar[par]), (uint32_t)(b >> 1) & 1u, abort_flag, S.status);
+                bool ok = !failed && (wt >= 32 || mbar_wait_cluster(smem_u32(&ctl.dbar[par]), (uint32_t)(b >> 1) & 1u, abort_flag, S.status));
                 if (wt < 32) fence_cluster(); // the walk's ordinary stores into this CTA's part of the model
                 ok = work_bar_and(ok);
                 if (!ok) { aborted = true; break; }
             } else {
-                bool ok = wt >= 32 || mbar_wait_cluster(smem_u32(&ctl.dbar[par]), (uint32_t)(b >> 1) & 1u, abort_flag, S.status);
+                bool ok = !failed && (wt >= 32 || mbar_wait_cluster(smem_u32(&ctl.dbar[par]), (uint32_t)(b >> 1) & 1u, abort_flag, S.status));
                 ok = work_bar_and(ok);
                 if (!ok) { aborted = true; break; }
                 LA_T(wd);
@@ -1522,16 +1512,21 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                 }
                 work_bar();
             }
-            mbar_arrive_expect_tx_if(smem_u32(&ctl.dbar[par]), (uint32_t)(kLB * 4), wt == 0); // for block b + 2
-            issue_sub(b + kSubSlots, dn); // block b's slot is free
+            if (b >= 0) {
+                mbar_arrive_expect_tx_if(smem_u32(&ctl.dbar[par]), (uint32_t)(kLB * 4), wt == 0); // for block b + 2
+                issue_sub(b + kSubSlots, dn); // block b's slot is free
+            }
             LA_T(ws);
-            // a block right behind a walked one starts from the model as the walk left it
-            if (sl0 && b + 1 < nb && !sl1) {
-                if (!take_dots(b + 1)) { aborted = true; break; }
+            // dot products: of block b + 2 against the model as it is now; of block b + 1 first if block b was walked in
+            // place (a block right behind a walked one starts from the model as the walk left it)
+#pragma unroll 1
+            for (int ahead = 1; ahead <= 2; ++ahead) {
+                // (one block ahead: block b + 1 after block b's update, whatever block b was)
+                const bool due = depth == 1 ? (ahead == 1 && b + 1 < nb && !sl1)
+                                            : (ahead == 1 ? (sl0 && b + 1 < nb && !sl1) : (b + 2 < nb && !sl2 && !sl1));
+                if (due && !take_dots(b + ahead)) { aborted = true; break; }
             }
-            if (b + 2 < nb && !sl2 && !sl1) {
-                if (!take_dots(b + 2)) { aborted = true; break; }
-            }
+            if (aborted) break;
             sl0 = sl1; sl1 = sl2; sl2 = sl3;
             sl3 = b + kSubSlots < nb && (dn[3] & 1u) != 0u;
             LA_T(wg);
@@ -1682,6 +1677,17 @@ template <int LOSS> cudaError_t launch_slices(Glm &g, std::vector<LookParams> &P
     const int S = (int)P.size(), R = g.la_regions;
     cudaError_t e = cudaMemsetAsync(g.la_cursor, 0, 4 * sizeof(unsigned long long), g.stream);
     if (e != cudaSuccess) return e;
+    if (!g.la_overlap) {
+        // the chains take most of the SMs: the prepare kernels get the whole GPU between the chain launches instead of
+        // the few SMs beside them
+        for (int s = 0; s < S && e == cudaSuccess; ++s) {
+            if (s > 0) e = cudaMemsetAsync(g.la_cursor + (s % R), 0, sizeof(unsigned long long), g.stream);
+            if (e == cudaSuccess) e = launch_prepare_on<LOSS>(g, P[s], g.stream);
+            if (s == 0 && g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
+            if (e == cudaSuccess) e = launch_chain_on<LOSS>(g, P[s]);
+        }
+        return e;
+    }
     e = launch_prepare_on<LOSS>(g, P[0], g.stream);
     if (e != cudaSuccess) return e;
     if (g.time_prepare) (void)cudaEventRecord(g.ev[4], g.stream);
@@ -1737,6 +1743,17 @@ void lookahead_plan(Glm &g, int32_t K)
         }
     }
     g.la_logC = logC;
+    // Beside chains on at most half of the SMs the prepare kernels keep up: they run on the side stream, and the chain
+    // looks two blocks ahead (the cross Gram matrices cost the prepare kernels 70 % more). Otherwise the prepare kernels
+    // alternate with the chain launches on the whole GPU, without the cross Gram matrices.
+    g.la_overlap = ((int64_t)K << logC) * 2 <= g.sm_count;
+    g.la_depth = g.la_overlap ? 2 : 1;
+    {
+        const char *env = getenv("CHICLE_LA_DEPTH");
+        if (env && (env[0] == '1' || env[0] == '2') && env[1] == 0) g.la_depth = env[0] - '0';
+        env = getenv("CHICLE_LA_OVERLAP");
+        if (env && (env[0] == '0' || env[0] == '1') && env[1] == 0) g.la_overlap = env[0] == '1';
+    }
     const size_t budget = (size_t)(g.max_smem_optin > 0 ? g.max_smem_optin : 227 * 1024);
     if (dense) {
         g.la_nzcap = 0;
@@ -1825,7 +1842,7 @@ cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
         const int n = forced > max_slices ? max_slices : forced;
         F.assign(1, 0.0);
         for (int s = 1; s <= n; ++s) F.push_back((double)s / n);
-    } else if (!g.la_stream || g.la_regions == 1 || max_nb < 512) {
+    } else if ((g.la_overlap && !g.la_stream) || g.la_regions == 1 || max_nb < 512) {
         F = {0.0, 1.0};
     } else {
         cap = 1.0 / 16;
@@ -1888,6 +1905,7 @@ cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
         p.blk_base = g.la_blk_base + (size_t)s * ((size_t)K + 1);
         p.K = K;
         p.logC = g.la_logC;
+        p.depth = g.la_depth;
         p.nzcap = g.la_nzcap;
         p.hotc = g.la_hotc;
         p.n_blocks = blocks[(size_t)s];

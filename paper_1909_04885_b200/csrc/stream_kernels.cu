@@ -476,7 +476,10 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
             fetch(t + step, rs_n, re_n, lab_n, sta_n);
             if (!gap_wait(smem_u32(&sm.full[st]), (uint32_t)(k / kGapStages) & 1u, abort_flag, status)) break;
             const int64_t base = sm.base[st];
-            double dot = 0.0;
+            // A coordinate's dot product is taken in fp32 (as the solvers take it), every thread its own entries in a
+            // fixed order, and enters the fp64 sums over the coordinates once: a conversion and an fp64 multiply-add
+            // per non-zero were what the kernel was bound by (instruction issue), not the memory traffic.
+            float dot = 0.0f;
             if (base >= 0) {
                 // staged: 32-bit offsets into the stage, every load unconditional (clamped) and the gathers beyond the
                 // staged head of the vector predicated, so that nothing branches per non-zero
@@ -504,21 +507,17 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
 #pragma unroll
                     for (int q = 0; q < kMaxPer; ++q) {
                         // (x is 0 beyond the coordinate's end; fp32 v - y for the staged head, as the solvers' residual)
-                        if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) {
-                            const double t = ii[q] >= hot_n ? (double)tt[q] - (double)yy[q] : (double)hh[q];
-                            dot = fma((double)xx[q], t, dot);
-                        } else {
-                            dot = fma((double)xx[q], (double)(ii[q] >= hot_n ? tt[q] : hh[q]), dot);
-                        }
+                        if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) dot = fmaf(xx[q], ii[q] >= hot_n ? tt[q] - yy[q] : hh[q], dot);
+                        else dot = fmaf(xx[q], ii[q] >= hot_n ? tt[q] : hh[q], dot);
                     }
                 }
             } else {
                 for (int64_t e = rs + sub; e < re; e += TPR) {
                     const int32_t i = indices[e];
-                    double t;
-                    if (i < hot_n) t = (double)sm.vhot[i];
-                    else t = (double)vec[i] - (LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? (double)labels[i] : 0.0);
-                    dot = fma((double)values[e], t, dot);
+                    float t;
+                    if (i < hot_n) t = sm.vhot[i];
+                    else t = vec[i] - (LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? labels[i] : 0.0f);
+                    dot = fmaf(values[e], t, dot);
                 }
             }
             // the stage is free once every lane of the warp has read its entries
@@ -526,7 +525,7 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
             if (lane == 0) mbar_arrive(smem_u32(&sm.empty[st]));
 #pragma unroll
             for (int o = 1; o < TPR; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            if (owner) gap_term<LOSS>(dot, lab, sta, inv_lam_n, s0, s1);
+            if (owner) gap_term<LOSS>((double)dot, lab, sta, inv_lam_n, s0, s1);
         }
     }
     // slice of the shared vector owned by this block (consumer threads)

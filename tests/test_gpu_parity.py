@@ -396,6 +396,20 @@ def test_lookahead_runs_are_bit_reproducible(name, scale, slices, monkeypatch):
     assert np.array_equal(res[0][0], res[1][0]) and np.array_equal(res[0][1], res[1][1]) and res[0][2] == res[1][2]
 
 
+@pytest.mark.parametrize("depth,overlap,cluster", [("1", "0", "1"), ("1", "1", "2"), ("2", "0", "4"), ("2", "1", "8")])
+def test_lookahead_depths_overlap_modes_and_cluster_sizes(depth, overlap, cluster, monkeypatch):
+    # dot products one or two blocks ahead of the recurrence, prepare kernels beside the chain kernels or alternating
+    # with them, 1 to 8 CTAs per partition: every combination walks the same order and must match the oracle
+    monkeypatch.setenv("CHICLE_LA_DEPTH", depth)
+    monkeypatch.setenv("CHICLE_LA_OVERLAP", overlap)
+    monkeypatch.setenv("CHICLE_LA_CLUSTER", cluster)
+    monkeypatch.setenv("CHICLE_LA_SLICES", "3")
+    run_parity(datagen.make("hinge_csr", 100), rounds=3)
+    run_parity(datagen.make("ridge_csc", 100), rounds=2)
+    run_parity(tiny_dense(700, 28, seed=2, loss="logistic", K=3), rounds=3)
+    run_parity(tiny_csr(200, 3000, seed=9, K=2, density=0.03, long_row=500), rounds=3)   # blocks walked in place
+
+
 def test_a_missing_record_ends_in_a_timeout_status_and_the_handle_stays_usable(monkeypatch):
     # Failure detection without a fault: one block's records are left unpublished (a host-side test aid), so the chain
     # kernel finds nothing to copy, sets the status word with no copy in flight, every wait in the cluster runs out
