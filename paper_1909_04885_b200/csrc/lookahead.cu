@@ -1743,11 +1743,14 @@ void lookahead_plan(Glm &g, int32_t K)
         }
     }
     g.la_logC = logC;
-    // Beside chains on at most half of the SMs the prepare kernels keep up: they run on the side stream, and the chain
-    // looks two blocks ahead (the cross Gram matrices cost the prepare kernels 70 % more). Otherwise the prepare kernels
-    // alternate with the chain launches on the whole GPU, without the cross Gram matrices.
+    // Beside chains on at most half of the SMs the prepare kernels run on the side stream; otherwise they alternate with
+    // the chain launches and have the whole GPU meanwhile (config 5, K = 128: 171 against 542 ms per round).
     g.la_overlap = ((int64_t)K << logC) * 2 <= g.sm_count;
-    g.la_depth = g.la_overlap ? 2 : 1;
+    // Two blocks ahead pays where the chains bound the round: dense rows (the recurrence itself is the cost) and sparse
+    // data with a cluster per partition. One CTA per partition on sparse data means many partitions: there the prepare
+    // kernels bound the round and run 40 % faster without the cross Gram matrices (measured on the hashed workload: K = 64
+    // 157 against 219 ms per round; K = 16 with four CTAs per partition 253 against 308 ms the other way round).
+    g.la_depth = (dense || logC >= 1) && g.la_overlap ? 2 : 1;
     {
         const char *env = getenv("CHICLE_LA_DEPTH");
         if (env && (env[0] == '1' || env[0] == '2') && env[1] == 0) g.la_depth = env[0] - '0';
