@@ -15,7 +15,11 @@
  *
  * Conventions
  *   - Every call returns a chicle_status_t. No C++ exception crosses this boundary. Out-parameters are left
- *     untouched on error. After any error other than CHICLE_ERR_CUDA the handle is unchanged and usable.
+ *     untouched on error. After any error other than CHICLE_ERR_CUDA the handle is usable, and unchanged with two
+ *     exceptions: a partition call that runs out of memory (CHICLE_ERR_OOM) has released the old per-partition
+ *     workspaces first (two of them do not fit at the largest problems) and leaves the handle without a partition,
+ *     alpha and v kept: call chicle_partition again; and a round that ended with CHICLE_ERR_TIMEOUT or
+ *     CHICLE_ERR_NUMERIC has left alpha and v part-way through the round (restore them with chicle_set_state).
  *   - All pointers named host_* are host memory; chicle_matrix_t says where its arrays live. The library copies
  *     what it needs at create time: the caller keeps ownership of everything it passes and may free it as soon
  *     as the call returns. Everything the library allocates is released by chicle_glm_destroy.
@@ -210,7 +214,9 @@ chicle_status_t chicle_get_permutation(chicle_glm_t *h, int64_t round, int32_t k
 
 /* Overwrite the state (checkpoint restore, or re-synchronising with an external trajectory). host_alpha has one
  * entry per coordinate; host_v may be NULL, in which case v is recomputed from alpha on the device
- * (v = X^T alpha, or X w). `round` >= 0 becomes the round counter. Synchronises. */
+ * (v = X^T alpha, or X w) with floating-point atomics, whose order of additions is not fixed: unlike everything else
+ * in the library, a v rebuilt this way (and what later rounds make of it) may differ in the last bits from run to run;
+ * pass host_v for bit-reproducible runs. `round` >= 0 becomes the round counter. Synchronises. */
 chicle_status_t chicle_set_state(chicle_glm_t *h, const float *host_alpha, const float *host_v, int64_t round);
 
 /* Current round counter, partition count and coordinate / shared-vector lengths; any pointer may be NULL. */

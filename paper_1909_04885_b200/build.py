@@ -36,7 +36,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("CHICLE_NVCC_FLAGS", "").split()  # e.g. -DCHICLE_LA_CHECK for the look-ahead solver's self-check build
+    cmd += os.environ.get("CHICLE_NVCC_FLAGS", "").split()  # e.g. -DCHICLE_LA_TIMING: cycle counters around the look-ahead solver's phases, printed after every launch
     cmd += ["-o", tmp] + sources()
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

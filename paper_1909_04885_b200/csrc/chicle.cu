@@ -441,12 +441,15 @@ static chicle_status_t partition_impl(chicle_glm_t *h, int32_t K, uint64_t seed,
     return CHICLE_OK;
 }
 
-chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed) { return partition_impl(h, K, seed, nullptr); }
+chicle_status_t chicle_partition(chicle_glm_t *h, int32_t K, uint64_t seed)
+{
+    try { return partition_impl(h, K, seed, nullptr); } catch (...) { return CHICLE_ERR_OOM; }
+}
 
 chicle_status_t chicle_partition_sizes(chicle_glm_t *h, int32_t K, uint64_t seed, const int64_t *host_sizes)
 {
     if (h && !host_sizes) return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_partition_sizes: sizes is NULL");
-    return partition_impl(h, K, seed, host_sizes);
+    try { return partition_impl(h, K, seed, host_sizes); } catch (...) { return CHICLE_ERR_OOM; }
 }
 
 chicle_status_t chicle_partition_chunks(chicle_glm_t *h, int32_t K, uint64_t seed, int64_t n_chunks, const int64_t *host_chunk_off,
@@ -454,7 +457,7 @@ chicle_status_t chicle_partition_chunks(chicle_glm_t *h, int32_t K, uint64_t see
 {
     if (!h) return CHICLE_ERR_INVALID_ARG;
     const ChunkPlacement cp{n_chunks, host_chunk_off, host_chunk_task};
-    return partition_impl(h, K, seed, nullptr, &cp);
+    try { return partition_impl(h, K, seed, nullptr, &cp); } catch (...) { return CHICLE_ERR_OOM; }
 }
 
 // One round. host_steps == nullptr: every partition takes H steps (0: one local epoch). Otherwise partition k takes
@@ -539,14 +542,14 @@ static chicle_status_t round_impl(chicle_glm_t *h, int64_t H, const int64_t *hos
 chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime, chicle_round_stats_t *stats)
 {
     if (!h) return CHICLE_ERR_INVALID_ARG;
-    return round_impl(h, H, nullptr, sigma_prime, stats);
+    try { return round_impl(h, H, nullptr, sigma_prime, stats); } catch (...) { return CHICLE_ERR_OOM; }
 }
 
 chicle_status_t chicle_cocoa_round_steps(chicle_glm_t *h, const int64_t *host_steps, float sigma_prime, chicle_round_stats_t *stats)
 {
     if (!h) return CHICLE_ERR_INVALID_ARG;
     if (!host_steps) return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_cocoa_round_steps: steps is NULL");
-    return round_impl(h, 0, host_steps, sigma_prime, stats);
+    try { return round_impl(h, 0, host_steps, sigma_prime, stats); } catch (...) { return CHICLE_ERR_OOM; }
 }
 
 chicle_status_t chicle_duality_gap(chicle_glm_t *h, double *host_gap, double *host_primal, double *host_dual)

@@ -30,7 +30,10 @@ extern "C" {
 
 int64_t chicle_chunks_cut(int64_t n_coord, const int64_t *host_indptr, int64_t dense_dim, int64_t chunk_bytes, int64_t *host_chunk_off)
 {
-    if (n_coord < 1 || !host_chunk_off || (!host_indptr && dense_dim < 1)) return -1;
+    if (n_coord < 1 || chunk_bytes < 1 || !host_chunk_off || (!host_indptr && dense_dim < 1)) return -1;
+    if (host_indptr)
+        for (int64_t i = 0; i < n_coord; ++i)
+            if (host_indptr[i + 1] < host_indptr[i]) return -1;
     int64_t C = 0, used = 0;
     host_chunk_off[0] = 0;
     for (int64_t i = 0; i < n_coord; ++i) {
@@ -47,6 +50,7 @@ int64_t chicle_chunks_cut(int64_t n_coord, const int64_t *host_indptr, int64_t d
 
 chicle_status_t chicle_chunks_assign(int64_t n_chunks, int32_t K, uint64_t seed, int32_t *host_chunk_task)
 {
+    try {
     if (K < 1 || (int64_t)K > n_chunks || !host_chunk_task) return CHICLE_ERR_INVALID_ARG;
     std::vector<int64_t> order((size_t)n_chunks);
     for (int64_t c = 0; c < n_chunks; ++c) order[(size_t)c] = c;
@@ -59,10 +63,12 @@ chicle_status_t chicle_chunks_assign(int64_t n_chunks, int32_t K, uint64_t seed,
         pos += m;
     }
     return CHICLE_OK;
+    } catch (...) { return CHICLE_ERR_OOM; }
 }
 
 chicle_status_t chicle_chunks_scale_in(int64_t n_chunks, int32_t K_old, int32_t K_new, int32_t *host_chunk_task)
 {
+    try {
     if (K_new < 1 || K_new > K_old || n_chunks < 1 || !host_chunk_task) return CHICLE_ERR_INVALID_ARG;
     int32_t next = 0;
     for (int64_t c = 0; c < n_chunks; ++c) {
@@ -72,10 +78,12 @@ chicle_status_t chicle_chunks_scale_in(int64_t n_chunks, int32_t K_old, int32_t 
         }
     }
     return CHICLE_OK;
+    } catch (...) { return CHICLE_ERR_OOM; }
 }
 
 chicle_status_t chicle_chunks_scale_out(int64_t n_chunks, int32_t K_old, int32_t K_new, uint64_t seed, int32_t *host_chunk_task)
 {
+    try {
     if (K_old < 1 || K_new < K_old || n_chunks < 1 || !host_chunk_task) return CHICLE_ERR_INVALID_ARG;
     const int32_t add = K_new - K_old;
     if (add == 0) return CHICLE_OK;
@@ -97,11 +105,13 @@ chicle_status_t chicle_chunks_scale_out(int64_t n_chunks, int32_t K_old, int32_t
         }
     }
     return CHICLE_OK;
+    } catch (...) { return CHICLE_ERR_OOM; }
 }
 
 int chicle_chunks_rebalance_step(int64_t n_chunks, const int64_t *host_chunk_off, int32_t K, const double *host_time_per_sample,
                                  int32_t *host_chunk_task)
 {
+    try {
     if (K < 1 || n_chunks < 1 || !host_chunk_off || !host_time_per_sample || !host_chunk_task) return -1;
     std::vector<int64_t> samples((size_t)K, 0);
     for (int64_t c = 0; c < n_chunks; ++c) {
@@ -124,6 +134,7 @@ int chicle_chunks_rebalance_step(int64_t n_chunks, const int64_t *host_chunk_off
     if (t_slow - t_fast <= one_chunk) return 0;
     host_chunk_task[last] = fast;
     return 1;
+    } catch (...) { return -1; }
 }
 
 } // extern "C"

@@ -27,6 +27,11 @@
 //                         through distributed shared memory by asynchronous stores that complete on the receiver's
 //                         mbarrier; no multicast, every wait bounded.
 //
+// Where many partitions leave the prepare kernels few SMs (one CTA per partition on sparse data), the dot products are
+// taken one block ahead only, against the model after the block before: no cross Gram matrix (the prepare kernels are
+// what bounds such rounds), and the recurrence warp waits for each block's dot products; and where the chains take more
+// than half of the SMs, the prepare kernels alternate with the chain launches instead of running beside them.
+//
 // A block with more non-zeros than the shared-memory buffers hold is flagged by the prepare kernel: the pipeline
 // drains, warp 0 of CTA 0 walks the block coordinate by coordinate against the whole model, and the pipeline starts
 // again behind it. Rounds that span several local epochs run the pair of kernels once per epoch.
