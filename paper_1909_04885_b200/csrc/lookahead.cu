@@ -122,6 +122,11 @@ struct LookParams {
     int32_t hotc;                // entry ids per CTA kept in shared memory
     int64_t n_blocks;
     int64_t drop_block;          // test aid: this block's records are left unpublished (-1: none)
+    int32_t model_in;            // the round's first chain launch: row k of the update workspace holds U_k and is turned
+                                 // into the local model w = v + sigma' U_k in place
+    int32_t model_out;           // the round's last chain launch: the row is turned back into U_k. Between a round's
+                                 // launches the row holds w itself: an id beyond the part in shared memory costs one
+                                 // gather instead of two, and nothing is rounded from launch to launch
 };
 
 #ifdef CHICLE_LA_TIMING
@@ -192,13 +197,6 @@ __device__ __forceinline__ float ldcg_if(const float *p, bool on)
 __device__ __forceinline__ void red_add_if(float *p, float v, bool on)
 {
     asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q red.global.add.f32 [%0], %1;\n\t}" ::"l"(p), "f"(v), "r"((uint32_t)on) : "memory");
-}
-__device__ __forceinline__ float ldca_if(const float *p, bool on)
-{
-    float v;
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\tmov.f32 %0, 0f00000000;\n\t@q ld.global.ca.f32 %0, [%1];\n\t}"
-                 : "=f"(v) : "l"(p), "r"((uint32_t)on) : "memory");
-    return v;
 }
 
 // The recurrence in the form the chain runs it. Every loss keeps one number s_j per coordinate that is linear in the
@@ -1062,8 +1060,13 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
     }
     for (int l = tid; l < hot_mine; l += kChainThreads) {
         const size_t g = ((size_t)l << logC) + crank;
-        W[l] = fmaf(sigma, Uk[g], S.vbase[g]);
+        W[l] = P.model_in ? fmaf(sigma, Uk[g], S.vbase[g]) : Uk[g];
     }
+    // the ids beyond the part in shared memory that fall to this CTA (id mod C): the model in place
+    const size_t cold0 = (size_t)hot_total + (((size_t)crank - (size_t)hot_total) & (size_t)(C - 1));
+    if (P.model_in)
+        for (size_t g = cold0 + ((size_t)tid << logC); g < (size_t)S.dim; g += (size_t)kChainThreads << logC)
+            Uk[g] = fmaf(sigma, Uk[g], S.vbase[g]);
     __syncthreads();
     cluster_arrive();
     cluster_wait();
@@ -1119,7 +1122,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                     for (int e = lane; e < n; e += 32) {
                         const uint32_t g = DENSE ? (uint32_t)e : (uint32_t)ix[e];
                         const float ww = g < hot_total ? ld_cluster_f32(mapa_u32(w_base + 4u * (g >> logC), g & (uint32_t)(C - 1)))
-                                                       : fmaf(sigma, __ldcg(Uk + g), S.vbase[g]);
+                                                       : __ldcg(Uk + g);
                         acc = fmaf(xv[e], ww, acc);
                     }
                     acc = warp_sum(acc);
@@ -1135,7 +1138,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                             if (g < hot_total) {
                                 const uint32_t a = mapa_u32(w_base + 4u * (g >> logC), g & (uint32_t)(C - 1));
                                 st_cluster_f32(a, fmaf(sigma * delta, xv[e], ld_cluster_f32(a)));
-                            } else Uk[g] = fmaf(delta, xv[e], __ldcg(Uk + g));
+                            } else Uk[g] = fmaf(sigma * delta, xv[e], __ldcg(Uk + g));
                         }
                     if (lane == 0) S.alpha[h.coord] = new_state;
                     __syncwarp();
@@ -1337,10 +1340,32 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                 // Eight threads per coordinate, each its every eighth non-zero: the first two with all loads issued
                 // before anything is used. Ids below hot_total from shared memory; the others from row k of the
                 // update workspace (read at L2: the updates are made there by reductions) and from v.
-                if (wt < kLB * 8) {
+                if (wt < kLB * 8 && hot_total == 0u) {
+                    // (no id in shared memory: every gather goes to L2, eight per thread in flight)
                     const int j = wt >> 3, qq = wt & 7;
                     const int lo = h.roff[j] + qq, hi = h.roff[j + 1];
-                    float x[2], hv[2], uu[2], vb[2];
+                    float acc = 0.0f;
+                    for (int e0 = lo; e0 < hi; e0 += 64) {
+                        float x8[8], u8[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int e = e0 + 8 * u;
+                            const bool on = e < hi;
+                            x8[u] = on ? val[e] : 0.0f;
+                            const uint32_t g = on ? (meta[e] & kIdMask) : 0u;
+                            u8[u] = ldcg_if(Uk + g, on);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) acc = fmaf(x8[u], u8[u], acc);
+                    }
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+                    if (qq == 0) st_async_f32(p_buf0 + (slot * (uint32_t)(kMaxC * kLB) + (uint32_t)j) * 4u, acc, p_bar0 + slot * 8u);
+                } else if (wt < kLB * 8) {
+                    const int j = wt >> 3, qq = wt & 7;
+                    const int lo = h.roff[j] + qq, hi = h.roff[j + 1];
+                    float x[2], hv[2], uu[2];
                     bool cold[2];
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
@@ -1351,14 +1376,13 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                         cold[u] = on && g >= hot_total;
                         hv[u] = W[cold[u] ? 0u : (g >> logC)];
                         uu[u] = ldcg_if(Uk + (cold[u] ? g : 0u), cold[u]);
-                        vb[u] = ldca_if(S.vbase + (cold[u] ? g : 0u), cold[u]);
                     }
-                    float acc = x[0] * (cold[0] ? fmaf(sigma, uu[0], vb[0]) : hv[0]);
-                    acc = fmaf(x[1], cold[1] ? fmaf(sigma, uu[1], vb[1]) : hv[1], acc);
+                    float acc = x[0] * (cold[0] ? uu[0] : hv[0]);
+                    acc = fmaf(x[1], cold[1] ? uu[1] : hv[1], acc);
                     // (longer coordinates: four at a time, again with all loads first: an id beyond the part of the
                     // model in shared memory costs a round trip to L2, which the four share)
                     for (int e0 = lo + 16; e0 < hi; e0 += 32) {
-                        float x4[4], h4[4], u4[4], v4[4];
+                        float x4[4], h4[4], u4[4];
                         bool c4[4];
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
@@ -1369,10 +1393,9 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                             c4[u] = on && g >= hot_total;
                             h4[u] = W[c4[u] ? 0u : (g >> logC)];
                             u4[u] = ldcg_if(Uk + (c4[u] ? g : 0u), c4[u]);
-                            v4[u] = ldca_if(S.vbase + (c4[u] ? g : 0u), c4[u]);
                         }
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) acc = fmaf(x4[u], c4[u] ? fmaf(sigma, u4[u], v4[u]) : h4[u], acc);
+                        for (int u = 0; u < 4; ++u) acc = fmaf(x4[u], c4[u] ? u4[u] : h4[u], acc);
                     }
                     acc += __shfl_xor_sync(0xffffffffu, acc, 1);
                     acc += __shfl_xor_sync(0xffffffffu, acc, 2);
@@ -1433,7 +1456,33 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                     //     their product delta_j * x at their place in the id's list. One store per non-zero, its
                     //     address chosen without a branch: the list place, the model word, or a word that nobody reads;
                     //     ids beyond the part in shared memory add to the workspace row instead.
-                    if (wt < kLB * 8) {
+                    if (wt < kLB * 8 && hot_total == 0u) {
+                        // (no id in shared memory: a list place or a reduction at L2, eight non-zeros per turn)
+                        const int j = wt >> 3, qq = wt & 7;
+                        const int lo = h.roff[j] + qq, hi = h.roff[j + 1];
+                        const float d = dl[j];
+                        const uint32_t a_prod = smem_u32(prod), a_sink = smem_u32(&ctl.sink[lane]);
+                        for (int e0 = lo; e0 < hi; e0 += 64) {
+                            uint32_t m8[8];
+                            float p8[8];
+                            int c8[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                const int e = e0 + 8 * u;
+                                const bool on = e < hi;
+                                m8[u] = on ? meta[e] : 0u;
+                                p8[u] = on ? d * val[e] : 0.0f;
+                                c8[u] = on ? cpos[e] : 0;
+                            }
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                const bool shared_id = (m8[u] >> 31) != 0u;
+                                sts_f32(shared_id ? a_prod + 4u * (uint32_t)c8[u] : a_sink, p8[u]);
+                                const bool far = !shared_id && p8[u] != 0.0f; // (beyond the coordinate's end p8 is 0)
+                                red_add_if(Uk + (far ? (m8[u] & kIdMask) : 0u), sigma * p8[u], far);
+                            }
+                        }
+                    } else if (wt < kLB * 8) {
                         const int j = wt >> 3, qq = wt & 7;
                         const int lo = h.roff[j] + qq, hi = h.roff[j + 1];
                         const float d = dl[j];
@@ -1462,7 +1511,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                             const uint32_t addr = !on[u] ? a_sink : (shared_id ? a_prod + 4u * (uint32_t)cp[u] : (hot ? a_w + 4u * (g >> logC) : a_sink));
                             sts_f32(addr, shared_id ? p[u] : fmaf(sigma, p[u], w2[u]));
                             const bool far = on[u] && !shared_id && !hot && p[u] != 0.0f;
-                            red_add_if(Uk + (far ? g : 0u), p[u], far); // a reduction at L2, nothing waits for it
+                            red_add_if(Uk + (far ? g : 0u), sigma * p[u], far); // a reduction at L2, nothing waits for it
                         }
                         for (int e = lo + 16; e < hi; e += 8) {
                             const uint32_t mm = meta[e];
@@ -1470,7 +1519,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                             const float pp = d * val[e];
                             if (mm & 0x80000000u) prod[cpos[e]] = pp;
                             else if (g < hot_total) W[g >> logC] = fmaf(sigma, pp, W[g >> logC]);
-                            else if (pp != 0.0f) atomicAdd(Uk + g, pp);
+                            else if (pp != 0.0f) atomicAdd(Uk + g, sigma * pp);
                         }
                     }
                     work_bar();
@@ -1511,7 +1560,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                         for (int u = 0; u < 2; ++u)
                             if (quarter == 0 && on[u] && sum[u] != 0.0f) {
                                 if (g3[u] < hot_total) W[g3[u] >> logC] = fmaf(sigma, sum[u], W[g3[u] >> logC]);
-                                else atomicAdd(Uk + g3[u], sum[u]);
+                                else atomicAdd(Uk + g3[u], sigma * sum[u]);
                             }
                     }
                 }
@@ -1542,14 +1591,19 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
             d[0] = wd; d[1] = ws; d[2] = wg; d[3] = ws1; d[4] = wg0; d[5] = wg1;
         }
 #endif
-        if (!aborted) {
-            work_bar();
-            const float inv_sigma = 1.0f / sigma;
-            for (int l = wt; l < hot_mine; l += kWorkThreads) {
-                const size_t g = ((size_t)l << logC) + crank;
-                Uk[g] = (W[l] - S.vbase[g]) * inv_sigma;
-            }
+    }
+    if (is_worker && !aborted) {
+        // the model goes back to row k: as it is, or after the round's last launch as the update U_k = (w - v) / sigma'
+        const int wt = (warp - 1 - (warp >> 2)) * 32 + lane;
+        work_bar();
+        const float inv_sigma = 1.0f / sigma;
+        for (int l = wt; l < hot_mine; l += kWorkThreads) {
+            const size_t g = ((size_t)l << logC) + crank;
+            Uk[g] = P.model_out ? (W[l] - S.vbase[g]) * inv_sigma : W[l];
         }
+        if (P.model_out)
+            for (size_t g = cold0 + ((size_t)wt << logC); g < (size_t)S.dim; g += (size_t)kWorkThreads << logC)
+                Uk[g] = (__ldcg(Uk + g) - S.vbase[g]) * inv_sigma;
     }
     if (is_worker || nb == 0) {
         if ((tid & 31) == 0) *reinterpret_cast<volatile int *>(&ctl.done) = 1;
@@ -1624,9 +1678,13 @@ template <int LOSS, int NZ, int HT, int THREADS> cudaError_t launch_prepare(cons
 }
 
 constexpr int kPreSmallNz = 2048;
+constexpr int kPreMidNz = 3072;
 
 // true: the prepare kernel with arrays for 2 048 non-zeros per block serves (32 coordinates of 50 on average, with room)
 bool small_prepare(const Glm &g) { return 32.0 * (double)g.nnz / (double)g.n_coord * 1.25 <= (double)kPreSmallNz; }
+// true: arrays for 3 072 non-zeros per block serve (two CTAs of 512 threads share an SM; with 4 096 it is one). Blocks
+// with more are walked in place either way unless a cluster shares them out.
+bool mid_prepare(const Glm &g) { return g.la_logC == 0 || 32.0 * (double)g.nnz / (double)g.n_coord * 1.1 <= (double)kPreMidNz; }
 
 // The prepare kernel of one launch's blocks on `stream`.
 template <int LOSS> cudaError_t launch_prepare_on(Glm &g, const LookParams &P, cudaStream_t stream)
@@ -1649,6 +1707,9 @@ template <int LOSS> cudaError_t launch_prepare_on(Glm &g, const LookParams &P, c
     if (small_prepare(g)) {
         const unsigned grid = stream == g.stream || nb < free_sms * 3 ? nb : free_sms * 3;
         e = launch_prepare<LOSS, kPreSmallNz, 2048, 256>(P, grid, stream);
+    } else if (mid_prepare(g)) {
+        const unsigned grid = stream == g.stream || nb < free_sms * 2 ? nb : free_sms * 2;
+        e = launch_prepare<LOSS, kPreMidNz, 4096, 512>(P, grid, stream);
     } else {
         const unsigned grid = stream == g.stream || nb < free_sms ? nb : free_sms;
         e = launch_prepare<LOSS, 4096, 4096, 512>(P, grid, stream);
@@ -1918,6 +1979,8 @@ cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
         p.hotc = g.la_hotc;
         p.n_blocks = blocks[(size_t)s];
         p.drop_block = (drop && s == 0) ? atoll(drop) : -1;
+        p.model_in = s == 0 ? 1 : 0;
+        p.model_out = s == Sn - 1 ? 1 : 0;
     }
     g.la_last_slices = Sn;
     g.solver_launches += 1 + 2 * Sn; // block tables, then a prepare and a chain launch per slice

@@ -410,6 +410,15 @@ def test_lookahead_depths_overlap_modes_and_cluster_sizes(depth, overlap, cluste
     run_parity(tiny_csr(200, 3000, seed=9, K=2, density=0.03, long_row=500), rounds=3)   # blocks walked in place
 
 
+@pytest.mark.parametrize("cluster", ["1", "2"])
+def test_ids_beyond_the_shared_memory_part_across_slices(cluster, monkeypatch):
+    # 25 000 or 50 000 features against some 21 600 model entries per CTA in shared memory: the rest of the local model
+    # lives in the partition's row of the update workspace, as the model itself between the launches of a round
+    monkeypatch.setenv("CHICLE_LA_CLUSTER", cluster)
+    monkeypatch.setenv("CHICLE_LA_SLICES", "3")
+    run_parity(datagen.make("hinge_csr", 4 if cluster == "1" else 2), rounds=2)
+
+
 def test_a_missing_record_ends_in_a_timeout_status_and_the_handle_stays_usable(monkeypatch):
     # Failure detection without a fault: one block's records are left unpublished (a host-side test aid), so the chain
     # kernel finds nothing to copy, sets the status word with no copy in flight, every wait in the cluster runs out
