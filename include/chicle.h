@@ -195,6 +195,38 @@ chicle_status_t chicle_cocoa_round(chicle_glm_t *h, int64_t H, float sigma_prime
 chicle_status_t chicle_cocoa_round_steps(chicle_glm_t *h, const int64_t *host_steps, float sigma_prime,
                                          chicle_round_stats_t *stats);
 
+/* ---- One job on several GPUs: the partitions spread over ranks, the shared vector replicated (Sec. 4.2 "Trainer and
+ * solver": every iteration the trainer merges the solvers' updates and broadcasts the model; Sec. 4.3: that exchange is
+ * one model-sized vector per task; Appendix "Example application"). Every rank creates a handle over the same data
+ * and calls chicle_partition with the same K and seed, so all ranks hold the same partition map, visiting orders and
+ * (in sparse formats) the same internal numbering of the entries. A rank then runs only the partitions it owns, the
+ * ranks exchange their summed updates (an all-gather of `dim` floats per rank, done by the caller with any collective
+ * library: the library itself never touches another GPU's memory), and every rank applies all of them in rank order.
+ *
+ * chicle_cocoa_round_delta: chicle_cocoa_round_steps (budget 0 for the partitions of other ranks), except that the sum
+ * of the partitions' updates, in ascending k with an fp64 accumulator, is written to dev_delta (a device array of
+ * `len` = length of the shared vector floats, in the library's internal order of the entries: only meaningful to
+ * chicle_apply_deltas of a handle over the same data) and v is left as it was. The round counter advances.
+ *
+ * chicle_apply_deltas: v += dev_deltas[0] + ... + dev_deltas[count - 1] (count vectors of `len` floats one behind the
+ * other on the device, added in that order with an fp64 accumulator; ridge: the residual is refreshed). Ranks that
+ * apply the same vectors in the same order keep bit-identical copies of v. With one rank, a round_delta followed by
+ * apply_deltas equals chicle_cocoa_round_steps up to one rounding per entry (the sum is rounded to fp32 before it
+ * is added).
+ *
+ * chicle_export_state_of / chicle_import_state: the per-coordinate state (alpha, or w for ridge) is only current on
+ * the rank that owns the coordinate's partition. export writes to dev_out (device, one float per coordinate) the
+ * state of the coordinates whose partition k has host_keep[k] != 0 (K bytes on the host, read during the call) and 0
+ * elsewhere; summing the ranks' exports (exact: one non-zero term per coordinate) gives the whole state, which import
+ * copies into the handle. Needed before chicle_duality_gap, chicle_get_alpha and before a new partition changes the
+ * ownership. All four calls are asynchronous on the handle's stream; bad arguments give CHICLE_ERR_INVALID_ARG with
+ * nothing enqueued. */
+chicle_status_t chicle_cocoa_round_delta(chicle_glm_t *h, const int64_t *host_steps, float sigma_prime, float *dev_delta,
+                                         int64_t len, chicle_round_stats_t *stats);
+chicle_status_t chicle_apply_deltas(chicle_glm_t *h, const float *dev_deltas, int32_t count, int64_t len);
+chicle_status_t chicle_export_state_of(chicle_glm_t *h, const uint8_t *host_keep, float *dev_out, int64_t len);
+chicle_status_t chicle_import_state(chicle_glm_t *h, const float *dev_state, int64_t len);
+
 /* Duality gap P(w(alpha)) - D(alpha) of the current state (Sec. 4.1, Sec. 5: the metric solvers report), with
  * fp64 accumulation in a fixed order. host_gap / host_primal / host_dual may each be NULL. Synchronises. */
 chicle_status_t chicle_duality_gap(chicle_glm_t *h, double *host_gap, double *host_primal, double *host_dual);

@@ -25,7 +25,8 @@ EXPORTED = ["chicle_glm_create", "chicle_partition", "chicle_cocoa_round", "chic
             "chicle_get_v", "chicle_get_partition", "chicle_get_permutation", "chicle_set_state", "chicle_get_info",
             "chicle_last_error", "chicle_glm_destroy", "chicle_partition_noalloc", "chicle_partition_sizes",
             "chicle_cocoa_round_steps", "chicle_chunks_cut", "chicle_chunks_assign", "chicle_chunks_scale_in",
-            "chicle_chunks_scale_out", "chicle_chunks_rebalance_step", "chicle_partition_chunks"]
+            "chicle_chunks_scale_out", "chicle_chunks_rebalance_step", "chicle_partition_chunks", "chicle_cocoa_round_delta",
+            "chicle_apply_deltas", "chicle_export_state_of", "chicle_import_state"]
 
 
 class ChicleError(RuntimeError):
@@ -77,6 +78,14 @@ def load():
     lib.chicle_cocoa_round.argtypes = [vp, i64, f32, C.POINTER(RoundStats)]
     lib.chicle_cocoa_round_steps.restype = C.c_int
     lib.chicle_cocoa_round_steps.argtypes = [vp, vp, f32, C.POINTER(RoundStats)]
+    lib.chicle_cocoa_round_delta.restype = C.c_int
+    lib.chicle_cocoa_round_delta.argtypes = [vp, vp, f32, vp, i64, C.POINTER(RoundStats)]
+    lib.chicle_apply_deltas.restype = C.c_int
+    lib.chicle_apply_deltas.argtypes = [vp, vp, i32, i64]
+    lib.chicle_export_state_of.restype = C.c_int
+    lib.chicle_export_state_of.argtypes = [vp, vp, vp, i64]
+    lib.chicle_import_state.restype = C.c_int
+    lib.chicle_import_state.argtypes = [vp, vp, i64]
     lib.chicle_chunks_cut.restype = i64
     lib.chicle_chunks_cut.argtypes = [i64, vp, i64, i64, vp]
     lib.chicle_chunks_assign.restype = C.c_int
@@ -265,6 +274,31 @@ class Glm:
                     "ms_prepare": rs.ms_prepare, "solver_slices": rs.solver_slices, "cluster_ctas": rs.cluster_ctas,
                     "solver_launches": rs.solver_launches, "order_launches": rs.order_launches}
         return None
+
+    def cocoa_round_delta(self, steps, sigma_prime: float, delta_out):
+        """``chicle_cocoa_round_delta``: the round with budgets ``steps``; the summed update goes to ``delta_out`` (a
+        CUDA tensor of ``dim`` floats on this handle's device) and v is left alone."""
+        st = np.ascontiguousarray(steps, np.int64)
+        if st.size != self.K:
+            raise ValueError("steps must have K entries")
+        self._check(self._lib.chicle_cocoa_round_delta(self._h, st.ctypes.data, C.c_float(float(sigma_prime)), _ptr(delta_out),
+                                                       delta_out.numel(), None))
+
+    def apply_deltas(self, deltas):
+        """``chicle_apply_deltas``: ``deltas`` is a contiguous CUDA tensor of shape (count, dim)."""
+        count = deltas.numel() // self.dim
+        self._check(self._lib.chicle_apply_deltas(self._h, _ptr(deltas), count, self.dim))
+
+    def export_state_of(self, keep, out):
+        """``chicle_export_state_of``: ``keep`` holds K flags, ``out`` is a CUDA tensor of one float per coordinate."""
+        kp = np.ascontiguousarray(keep, np.uint8)
+        if kp.size != self.K:
+            raise ValueError("keep must have K entries")
+        self._check(self._lib.chicle_export_state_of(self._h, kp.ctypes.data, _ptr(out), out.numel()))
+
+    def import_state(self, state):
+        """``chicle_import_state``: ``state`` is a CUDA tensor of one float per coordinate."""
+        self._check(self._lib.chicle_import_state(self._h, _ptr(state), state.numel()))
 
     def fail_allocations(self, on: bool):
         """Makes the allocator callback that the library was given refuse every request (return NULL) from now on, or

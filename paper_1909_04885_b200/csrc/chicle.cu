@@ -462,7 +462,9 @@ chicle_status_t chicle_partition_chunks(chicle_glm_t *h, int32_t K, uint64_t see
 
 // One round. host_steps == nullptr: every partition takes H steps (0: one local epoch). Otherwise partition k takes
 // host_steps[k] steps (H is 0 then).
-static chicle_status_t round_impl(chicle_glm_t *h, int64_t H, const int64_t *host_steps, float sigma_prime, chicle_round_stats_t *stats)
+// delta_out != nullptr: the summed update goes there (device, dim floats) and v stays as it is.
+static chicle_status_t round_impl(chicle_glm_t *h, int64_t H, const int64_t *host_steps, float sigma_prime, chicle_round_stats_t *stats,
+                                  float *delta_out = nullptr)
 {
     if (h->K <= 0) return fail(h, CHICLE_ERR_BAD_STATE, "chicle_partition must be called before chicle_cocoa_round");
     if (H < 0) return fail(h, CHICLE_ERR_INVALID_ARG, "H must be >= 0");
@@ -509,7 +511,7 @@ static chicle_status_t round_impl(chicle_glm_t *h, int64_t H, const int64_t *hos
     h->round_steps = nullptr;
     if (e != cudaSuccess) return fail_cuda(h, e, "local solver launch");
     if (stats) (void)cudaEventRecord(h->ev[2], s);
-    e = launch_reduce(*h);
+    e = delta_out ? launch_sum_updates(*h, delta_out) : launch_reduce(*h);
     if (e != cudaSuccess) return fail_cuda(h, e, "aggregation launch");
     if (stats) (void)cudaEventRecord(h->ev[3], s);
     h->round += 1;
@@ -550,6 +552,52 @@ chicle_status_t chicle_cocoa_round_steps(chicle_glm_t *h, const int64_t *host_st
     if (!h) return CHICLE_ERR_INVALID_ARG;
     if (!host_steps) return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_cocoa_round_steps: steps is NULL");
     try { return round_impl(h, 0, host_steps, sigma_prime, stats); } catch (...) { return CHICLE_ERR_OOM; }
+}
+
+chicle_status_t chicle_cocoa_round_delta(chicle_glm_t *h, const int64_t *host_steps, float sigma_prime, float *dev_delta, int64_t len,
+                                         chicle_round_stats_t *stats)
+{
+    if (!h) return CHICLE_ERR_INVALID_ARG;
+    if (!host_steps || !dev_delta || len != h->dim)
+        return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_cocoa_round_delta: steps or delta is NULL, or len is not the shared vector's length");
+    try { return round_impl(h, 0, host_steps, sigma_prime, stats, dev_delta); } catch (...) { return CHICLE_ERR_OOM; }
+}
+
+chicle_status_t chicle_apply_deltas(chicle_glm_t *h, const float *dev_deltas, int32_t count, int64_t len)
+{
+    if (!h) return CHICLE_ERR_INVALID_ARG;
+    if (!dev_deltas || count < 1 || len != h->dim)
+        return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_apply_deltas: deltas is NULL, count < 1, or len is not the shared vector's length");
+    cudaError_t e = cudaSetDevice(h->device);
+    if (e == cudaSuccess) e = launch_apply_deltas(*h, dev_deltas, count);
+    if (e != cudaSuccess) return fail_cuda(h, e, "chicle_apply_deltas");
+    return CHICLE_OK;
+}
+
+chicle_status_t chicle_export_state_of(chicle_glm_t *h, const uint8_t *host_keep, float *dev_out, int64_t len)
+{
+    if (!h) return CHICLE_ERR_INVALID_ARG;
+    if (h->K <= 0) return fail(h, CHICLE_ERR_BAD_STATE, "chicle_export_state_of needs a partition");
+    if (!host_keep || !dev_out || len != h->n_coord)
+        return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_export_state_of: keep or out is NULL, or len is not the number of coordinates");
+    cudaError_t e = cudaSetDevice(h->device);
+    // (the K words of the step budgets are free between rounds: the K bytes travel through them)
+    unsigned char *d_keep = reinterpret_cast<unsigned char *>(h->d_steps);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_keep, host_keep, (size_t)h->K, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = launch_mask_state(*h, d_keep, dev_out);
+    if (e != cudaSuccess) return fail_cuda(h, e, "chicle_export_state_of");
+    return CHICLE_OK;
+}
+
+chicle_status_t chicle_import_state(chicle_glm_t *h, const float *dev_state, int64_t len)
+{
+    if (!h) return CHICLE_ERR_INVALID_ARG;
+    if (!dev_state || len != h->n_coord)
+        return fail(h, CHICLE_ERR_INVALID_ARG, "chicle_import_state: state is NULL or len is not the number of coordinates");
+    cudaError_t e = cudaSetDevice(h->device);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->alpha, dev_state, (size_t)len * 4, cudaMemcpyDeviceToDevice, h->stream);
+    if (e != cudaSuccess) return fail_cuda(h, e, "chicle_import_state");
+    return CHICLE_OK;
 }
 
 chicle_status_t chicle_duality_gap(chicle_glm_t *h, double *host_gap, double *host_primal, double *host_dual)

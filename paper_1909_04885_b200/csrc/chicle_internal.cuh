@@ -143,6 +143,9 @@ cudaError_t launch_partition_chunks(Glm &g, int32_t K, int64_t C, const int64_t 
 cudaError_t launch_permutation(Glm &g, int64_t round, int64_t epochs);    // fills perm[epochs * n_coord]
 cudaError_t launch_local_solver(Glm &g, int64_t H, float sigma_prime, int *variant);
 cudaError_t launch_reduce(Glm &g);                                        // v += sum_k U_k ; U = 0 ; resid
+cudaError_t launch_sum_updates(Glm &g, float *delta);                     // delta = sum_k U_k ; U = 0 (v untouched)
+cudaError_t launch_apply_deltas(Glm &g, const float *deltas, int count);  // v += sum_g deltas[g] ; resid
+cudaError_t launch_mask_state(Glm &g, const unsigned char *keep, float *out); // out = state where keep[owner], else 0
 cudaError_t launch_gap(Glm &g);                                           // fills gap_out[0..2]
 cudaError_t launch_shared_vector(Glm &g);                                 // v = X^T alpha (or X w) from scratch
 cudaError_t launch_refresh_resid(Glm &g);                                 // ridge: resid = v - y

@@ -121,6 +121,50 @@ k_reduce_updates(float *__restrict__ v, float *__restrict__ U, int K, int64_t di
     }
 }
 
+// The same aggregation with the sum kept apart from v: delta[j] = sum_k U[k][j] (k ascending, fp64 accumulator), U
+// cleared, v untouched. What a rank of a job spread over several GPUs hands to the others (Sec. 4.2: the trainer merges
+// the solvers' updates and broadcasts the model).
+__global__ void __launch_bounds__(kThreads)
+k_sum_updates(float *__restrict__ U, int K, int64_t dim, float *__restrict__ delta)
+{
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < dim; i += (int64_t)gridDim.x * blockDim.x) {
+        double acc = 0.0;
+#pragma unroll 16
+        for (int k = 0; k < K; ++k) {
+            float *p = U + (size_t)k * dim + i;
+            acc += *p;
+            *p = 0.f;
+        }
+        delta[i] = (float)acc;
+    }
+}
+
+// v[j] += sum_g D[g][j] (g ascending, fp64 accumulator): the merged update of `count` ranks, each rank's vector `dim`
+// long and the vectors one behind the other; every rank adds them in the same order, so the replicas of v stay equal
+// bit for bit. Ridge: the residual is refreshed in the same pass.
+__global__ void __launch_bounds__(kThreads)
+k_apply_deltas(float *__restrict__ v, const float *__restrict__ D, int count, int64_t dim, const float *__restrict__ y,
+               float *__restrict__ resid)
+{
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < dim; i += (int64_t)gridDim.x * blockDim.x) {
+        double acc = v[i];
+        for (int g = 0; g < count; ++g) acc += D[(size_t)g * dim + i];
+        const float o = (float)acc;
+        v[i] = o;
+        if (resid) resid[i] = o - y[i];
+    }
+}
+
+// out[i] = keep[owner[i]] ? state[i] : 0: the part of the per-coordinate state that the partitions marked in `keep`
+// own (K bytes on the device).
+__global__ void __launch_bounds__(kThreads)
+k_mask_state(const float *__restrict__ state, const int32_t *__restrict__ owner, const unsigned char *__restrict__ keep,
+             int64_t n, float *__restrict__ out)
+{
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = keep[owner[i]] ? state[i] : 0.0f;
+}
+
 __global__ void k_resid(const float *__restrict__ v, const float *__restrict__ y, int64_t n, float *__restrict__ r)
 {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
@@ -664,6 +708,32 @@ cudaError_t launch_reduce(Glm &g)
         if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
         k_reduce_updates<1><<<grid, kThreads, 0, g.stream>>>(g.v, g.U, g.K, g.dim, y, resid);
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sum_updates(Glm &g, float *delta)
+{
+    unsigned grid = blocks_for(g.dim, kThreads);
+    if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
+    k_sum_updates<<<grid, kThreads, 0, g.stream>>>(g.U, g.K, g.dim, delta);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_apply_deltas(Glm &g, const float *deltas, int count)
+{
+    const float *y = g.loss == CHICLE_LOSS_RIDGE_PRIMAL ? g.labels : nullptr;
+    float *resid = g.loss == CHICLE_LOSS_RIDGE_PRIMAL ? g.resid : nullptr;
+    unsigned grid = blocks_for(g.dim, kThreads);
+    if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
+    k_apply_deltas<<<grid, kThreads, 0, g.stream>>>(g.v, deltas, count, g.dim, y, resid);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mask_state(Glm &g, const unsigned char *keep, float *out)
+{
+    unsigned grid = blocks_for(g.n_coord, kThreads);
+    if (grid > (unsigned)g.sm_count * 16) grid = (unsigned)g.sm_count * 16;
+    k_mask_state<<<grid, kThreads, 0, g.stream>>>(g.alpha, g.owner, keep, g.n_coord, out);
     return cudaGetLastError();
 }
 
