@@ -1,5 +1,5 @@
 #!/usr/bin/env python
-"""Benchmark of the CoCoA round on one B200 (or N independent replicas on N GPUs).
+"""Benchmark of the CoCoA round on one B200 (or one job spread over N GPUs: partitions k mod N on rank k).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--configs 4,1,2,3,5]
 
@@ -68,7 +68,8 @@ def describe(w, cfg, n_gpus):
             "n": w.n_rows, "d": w.n_cols, "nnz": w.nnz, "H": "one local epoch",
             "l2": "inputs (%.0f MB) %s the 126 MB L2%s" % (data_mb, "larger than" if data_mb > 126 else "smaller than",
                                                           "" if data_mb > 126 else ": every round also rewrites the K x d update rows and the solver's records"),
-            "parallelism": "1 GPU" if n_gpus == 1 else "%d independent replicas, no collective" % n_gpus}
+            "parallelism": "1 GPU" if n_gpus == 1 else "one job on %d GPUs: rank g runs the partitions k mod %d = g; one all-gather of the "
+                           "summed updates per round, one all-reduce of the per-coordinate state per gap evaluation" % (n_gpus, n_gpus)}
 
 
 def algorithmic_bytes_per_round(w):
@@ -140,9 +141,10 @@ def max_over_ranks(dist, value, device=None):
     return float(t.item())
 
 
-def aggregate(units_per_rank, world, seconds_max):
-    """Whole-job throughput: the units all ranks processed divided by the slowest rank's time."""
-    return units_per_rank * world / seconds_max
+def throughput(units, seconds_max):
+    """Whole-job throughput: the units the job processed divided by the slowest rank's time (with several ranks the
+    job is one: its units are not multiplied by the number of ranks)."""
+    return units / seconds_max
 
 
 def read_profile_numbers():
@@ -249,7 +251,13 @@ def run_config(cfg, w, steps, warmup, local, dist, dev, world, peaks, want_ttg, 
     from paper_1909_04885_b200 import binding
     comp_bytes, eff_bytes = algorithmic_bytes_per_round(w)
     bounds = schedule(w, steps)
-    glm = binding.from_workload(w, device=local, on_device=True)
+    handle = binding.from_workload(w, device=local, on_device=True)
+    glm = handle
+    if world > 1:
+        # one job over the ranks: every rank holds the data and the replicated shared vector and runs the partitions
+        # k mod world; the summed updates are exchanged once per round (strong scaling: the work is fixed)
+        from paper_1909_04885_b200 import sharded
+        glm = sharded.ShardedGlm(sharded.GlmBackend(handle), sharded.Comm(dist))
     ph0 = w.phases[0]
     glm.partition(ph0.K, ph0.seed)
     for _ in range(warmup):
@@ -287,8 +295,8 @@ def run_config(cfg, w, steps, warmup, local, dist, dev, world, peaks, want_ttg, 
     if dist is not None:
         dist.barrier()
     ms_max = max_over_ranks(dist, ms, dev)
-    value = aggregate(w.n_coord * steps, world, ms_max / 1e3)
-    glm.close()
+    value = throughput(w.n_coord * steps, ms_max / 1e3)
+    handle.close()
 
     def mean(key, sel=None):
         xs = [s[key] for s, K in zip(stats, Ks) if sel is None or K == sel]
@@ -365,16 +373,20 @@ def run_e2e(w, n_steps, local, dist, dev, world):
         t0 = time.perf_counter()
         g2 = binding.Glm(w.loss, w.fmt, w.n_rows, w.n_cols, pinned[0], pinned[1], w.lam,
                          pinned[2] if len(pinned) > 2 else None, pinned[3] if len(pinned) > 2 else None, device=local)
-        g2.partition(ph.K, ph.seed)
-        g2.cocoa_round(w.H, ph.sigma_prime)
-        g2.duality_gap()
+        job = g2
+        if world > 1:   # the same job over the ranks (every rank uploads the data and keeps a replica of v)
+            from paper_1909_04885_b200 import sharded
+            job = sharded.ShardedGlm(sharded.GlmBackend(g2), sharded.Comm(dist))
+        job.partition(ph.K, ph.seed)
+        job.cocoa_round(w.H, ph.sigma_prime)
+        job.duality_gap()
         g2.get_v(v_host)
         torch.cuda.synchronize()
         if it > 0:
             times.append(1e3 * (time.perf_counter() - t0))
         g2.close()
     e2e_max = max_over_ranks(dist, statistics.mean(times), dev)
-    return {"value": aggregate(w.n_coord, world, e2e_max / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": throughput(w.n_coord, e2e_max / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": e2e_max,
             "what": "create from pinned host arrays + partition (K=%d) + one round + gap + read-back of v, per step" % ph.K}
 
@@ -444,7 +456,7 @@ def run_b200(args):
                               "(measured with cycle counters in the recurrence warp, see profiles/)"}
     traffic = prof["traffic_bytes_per_step"] * n_head if (prof["traffic_bytes_per_step"] and args.scale == 1 and head == HEADLINE) else None
     line = {"metric": METRIC, "value": H["value"], "unit": UNIT, "n_gpus": world, "steps": H["steps"], "warmup": warmup,
-            "ms_per_step": H["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": H["ms_per_step"], "higher_is_better": True, "scaling": "weak" if world == 1 else "strong", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic", "config": H["config"], "clocks": H["clocks"], "e2e": e2e,
             "gpu_launches": H["gpu_launches"],
             "roofline": {"bound": "hbm", "kernel": "k_lookahead_chain at %s (local SCD solvers: one thread-block cluster per partition)" % dom_key,

@@ -122,6 +122,13 @@ def load():
     return lib
 
 
+def _stats_dict(rs) -> dict:
+    return {"ms_permutation": rs.ms_permutation, "ms_local": rs.ms_local, "ms_reduce": rs.ms_reduce,
+            "ms_total": rs.ms_total, "steps": rs.steps, "solver_variant": rs.solver_variant,
+            "ms_prepare": rs.ms_prepare, "solver_slices": rs.solver_slices, "cluster_ctas": rs.cluster_ctas,
+            "solver_launches": rs.solver_launches, "order_launches": rs.order_launches}
+
+
 def _is_torch(x) -> bool:
     return x is not None and type(x).__module__.startswith("torch")
 
@@ -268,21 +275,18 @@ class Glm:
             self._check(self._lib.chicle_cocoa_round_steps(self._h, st.ctypes.data, C.c_float(sp), ref))
         else:
             self._check(self._lib.chicle_cocoa_round(self._h, H, C.c_float(sp), ref))
-        if stats:
-            return {"ms_permutation": rs.ms_permutation, "ms_local": rs.ms_local, "ms_reduce": rs.ms_reduce,
-                    "ms_total": rs.ms_total, "steps": rs.steps, "solver_variant": rs.solver_variant,
-                    "ms_prepare": rs.ms_prepare, "solver_slices": rs.solver_slices, "cluster_ctas": rs.cluster_ctas,
-                    "solver_launches": rs.solver_launches, "order_launches": rs.order_launches}
-        return None
+        return _stats_dict(rs) if stats else None
 
-    def cocoa_round_delta(self, steps, sigma_prime: float, delta_out):
+    def cocoa_round_delta(self, steps, sigma_prime: float, delta_out, stats: bool = False):
         """``chicle_cocoa_round_delta``: the round with budgets ``steps``; the summed update goes to ``delta_out`` (a
         CUDA tensor of ``dim`` floats on this handle's device) and v is left alone."""
         st = np.ascontiguousarray(steps, np.int64)
         if st.size != self.K:
             raise ValueError("steps must have K entries")
+        rs = RoundStats() if stats else None
         self._check(self._lib.chicle_cocoa_round_delta(self._h, st.ctypes.data, C.c_float(float(sigma_prime)), _ptr(delta_out),
-                                                       delta_out.numel(), None))
+                                                       delta_out.numel(), C.byref(rs) if stats else None))
+        return _stats_dict(rs) if stats else None
 
     def apply_deltas(self, deltas):
         """``chicle_apply_deltas``: ``deltas`` is a contiguous CUDA tensor of shape (count, dim)."""

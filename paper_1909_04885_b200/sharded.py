@@ -78,6 +78,7 @@ class GlmBackend:
         import torch
         self.glm = glm
         self.device = torch.device("cuda", glm.device)
+        self.last_stats = None
         self._delta = torch.empty(glm.dim, dtype=torch.float32, device=self.device)
         self._state = torch.empty(glm.n_coord, dtype=torch.float32, device=self.device)
 
@@ -87,8 +88,8 @@ class GlmBackend:
     def partition_sizes(self) -> np.ndarray:
         return np.bincount(self.glm.get_partition(), minlength=self.glm.K).astype(np.int64)
 
-    def round_delta(self, budgets, sigma_prime: float):
-        self.glm.cocoa_round_delta(budgets, sigma_prime, self._delta)
+    def round_delta(self, budgets, sigma_prime: float, stats: bool = False):
+        self.last_stats = self.glm.cocoa_round_delta(budgets, sigma_prime, self._delta, stats=stats)
         return self._delta
 
     def apply_deltas(self, stacked):
@@ -129,17 +130,19 @@ class ShardedGlm:
         self.K = K
         self.sizes = self.backend.partition_sizes()
 
-    def cocoa_round(self, H: int = 0, sigma_prime: Optional[float] = None, steps=None):
+    def cocoa_round(self, H: int = 0, sigma_prime: Optional[float] = None, steps=None, stats: bool = False):
+        """One round of the whole job. `stats`: returns this rank's round statistics (a backend that keeps them)."""
         if self.K <= 0:
             raise RuntimeError("partition first")
         sp = float(self.K if sigma_prime is None else sigma_prime)
         budgets = shard_budgets(self.sizes, self.rank, self.world, H, steps)
-        delta = self.backend.round_delta(budgets, sp)
+        delta = self.backend.round_delta(budgets, sp, stats=True) if stats else self.backend.round_delta(budgets, sp)
         self.backend.sync()
         stacked = self.comm.all_gather(delta)
         self.backend.apply_deltas(stacked)
         self.backend.sync()  # `stacked` must outlive the kernel that reads it
         self._state_current = self.world == 1
+        return getattr(self.backend, "last_stats", None) if stats else None
 
     def sync_state(self):
         """Every rank receives the per-coordinate state of the coordinates it does not own."""

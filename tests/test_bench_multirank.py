@@ -1,4 +1,4 @@
-"""Host-side logic of bench.py for N > 1 (independent replicas, max-over-ranks timing), run as two gloo ranks on CPU."""
+"""Host-side logic of bench.py for N > 1 (one job over the ranks, timed by the slowest rank), run as two gloo ranks on CPU."""
 import os
 import sys
 
@@ -19,14 +19,14 @@ def _worker(rank, world, port, out):
     try:
         my_ms = 10.0 + 5.0 * rank                      # rank 1 is the slow one
         slowest = bench.max_over_ranks(dist, my_ms)
-        value = bench.aggregate(1000, world, slowest / 1e3)
+        value = bench.throughput(1000, slowest / 1e3)
         out[rank] = (slowest, value)
         dist.barrier()
     finally:
         dist.destroy_process_group()
 
 
-def test_replicas_are_timed_by_the_slowest_rank():
+def test_the_job_is_timed_by_the_slowest_rank():
     world = 2
     port = 29500 + os.getpid() % 2000
     with mp.Manager() as m:
@@ -36,13 +36,13 @@ def test_replicas_are_timed_by_the_slowest_rank():
     assert res[0] == res[1]
     slowest, value = res[0]
     assert slowest == 15.0
-    assert value == pytest.approx(2 * 1000 / 0.015)
+    assert value == pytest.approx(1000 / 0.015)
 
 
 def test_single_process_helpers():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.max_over_ranks(None, 3.5) == 3.5
-    assert bench.aggregate(10, 1, 2.0) == 5.0
+    assert bench.throughput(10, 2.0) == 5.0
     args = bench.parse_args([])
     assert args.gpus == 1 and args.steps >= 1 and args.warmup >= 3
