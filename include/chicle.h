@@ -25,6 +25,9 @@
  *     as the call returns. Everything the library allocates is released by chicle_glm_destroy.
  *   - One handle is bound to one device and one stream, and is not thread-safe. Calls enqueue work on that
  *     stream; calls that return host scalars or copy to host memory synchronise the stream.
+ *   - CHICLE_LOG=1 in the environment (read once per process): every failed call writes its message, and every
+ *     round one line with its step count, solver variant, launches and phase times, to stderr; a round is then
+ *     synchronised for its timings.
  *   - Kernels never trap. A device-side problem (a bounded wait that ran out, a non-finite step) is recorded in a
  *     status word that the next synchronising call returns as CHICLE_ERR_TIMEOUT / CHICLE_ERR_NUMERIC.
  *   - State machine (paper Sec. 3, ownership contract: data moves only between iterations):

@@ -22,10 +22,22 @@ namespace {
 
 thread_local std::string g_create_error;
 
+// CHICLE_LOG=1 in the environment: every failed call and every round writes a line to stderr (a round is then
+// synchronised for its timings, like a round that was asked for statistics).
+int log_level()
+{
+    static const int level = [] {
+        const char *env = getenv("CHICLE_LOG");
+        return env ? atoi(env) : 0;
+    }();
+    return level;
+}
+
 chicle_status_t fail(chicle_glm *h, chicle_status_t st, const std::string &msg)
 {
     if (h) h->err = msg;
     else g_create_error = msg;
+    if (log_level() >= 1) fprintf(stderr, "[chicle] error %d: %s\n", (int)st, msg.c_str());
     return st;
 }
 
@@ -466,6 +478,9 @@ chicle_status_t chicle_partition_chunks(chicle_glm_t *h, int32_t K, uint64_t see
 static chicle_status_t round_impl(chicle_glm_t *h, int64_t H, const int64_t *host_steps, float sigma_prime, chicle_round_stats_t *stats,
                                   float *delta_out = nullptr)
 {
+    chicle_round_stats_t log_stats;
+    const bool logging = log_level() >= 1;
+    if (logging && !stats) stats = &log_stats;
     if (h->K <= 0) return fail(h, CHICLE_ERR_BAD_STATE, "chicle_partition must be called before chicle_cocoa_round");
     if (H < 0) return fail(h, CHICLE_ERR_INVALID_ARG, "H must be >= 0");
     if (!(sigma_prime > 0.0f) || !(sigma_prime < 3.0e38f)) return fail(h, CHICLE_ERR_INVALID_ARG, "sigma_prime must be positive and finite");
@@ -537,6 +552,11 @@ static chicle_status_t round_impl(chicle_glm_t *h, int64_t H, const int64_t *hos
         r.solver_launches = steps > 0 ? (h->solver_launches > 0 ? h->solver_launches : 1) : 0;
         r.order_launches = (int32_t)(epochs * (22 + 5 * (h->K <= 256 ? 1 : 2)));
         *stats = r;
+        if (logging)
+            fprintf(stderr, "[chicle] round %lld: K=%d steps=%lld solver=%d slices=%d ctas/partition=%d launches=%d; ms: orders %.3f, "
+                    "local solvers %.3f (first prepare %.3f), aggregation %.3f\n", (long long)(h->round - 1), (int)h->K,
+                    (long long)r.steps, (int)r.solver_variant, (int)r.solver_slices, (int)r.cluster_ctas,
+                    (int)(r.solver_launches + r.order_launches + 1), r.ms_permutation, r.ms_local, r.ms_prepare, r.ms_reduce);
     }
     return CHICLE_OK;
 }

@@ -59,3 +59,22 @@ def test_create_without_a_gpu_fails_loudly(lib):
         binding.Glm("hinge", "dense", 2, 2, np.ones(4, np.float32), np.ones(2, np.float32), 0.1,
                     torch_allocator=False, stream=0)
     assert ei.value.status == 4 and "no host path" in str(ei.value)
+
+
+def test_errors_are_logged_when_asked(lib):
+    # CHICLE_LOG=1: a failed call writes a line to stderr (the variable is read once, so in a process of its own)
+    import subprocess
+    import sys
+    code = ("import ctypes, numpy as np\n"
+            "from paper_1909_04885_b200 import binding\n"
+            "lib = binding.load()\n"
+            "h = ctypes.c_void_p(); vals = np.ones(4, np.float32); y = np.ones(2, np.float32)\n"
+            "m = binding.Matrix(0, 0, 2, 2, 0, 2, None, None, vals.ctypes.data_as(ctypes.c_void_p))\n"
+            "st = lib.chicle_glm_create(ctypes.byref(m), y.ctypes.data_as(ctypes.c_void_p), ctypes.c_float(-1.0), 0, 0, None, None, ctypes.byref(h))\n"
+            "assert st == 1\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    for level, expect in (("1", True), ("0", False)):
+        env = dict(os.environ, CHICLE_LOG=level, PYTHONPATH=root)
+        r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+        assert r.returncode == 0, r.stderr
+        assert ("[chicle] error 1" in r.stderr and "lambda" in r.stderr) == expect
