@@ -55,7 +55,9 @@ typedef enum {
     CHICLE_ERR_CUDA = 4,
     CHICLE_ERR_UNSUPPORTED = 5,
     CHICLE_ERR_NUMERIC = 6,
-    CHICLE_ERR_TIMEOUT = 7
+    CHICLE_ERR_TIMEOUT = 7,
+    CHICLE_ERR_INTERNAL = 8 /* only from a library built with -DCHICLE_DEBUG_BOUNDS: an index that a kernel loaded lay
+                               outside its array; the access was skipped, the state is part-way through the call */
 } chicle_status_t;
 
 typedef enum { CHICLE_LOSS_HINGE_DUAL = 0, CHICLE_LOSS_LOGISTIC_DUAL = 1, CHICLE_LOSS_RIDGE_PRIMAL = 2 } chicle_loss_t;

@@ -15,8 +15,9 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("CHICLE_LIB_PATH") or os.path.join(_HERE, "libchicle.so")
 
-OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED, ERR_NUMERIC, ERR_TIMEOUT = range(8)
-STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_STATE", 3: "OOM", 4: "CUDA", 5: "UNSUPPORTED", 6: "NUMERIC", 7: "TIMEOUT"}
+OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED, ERR_NUMERIC, ERR_TIMEOUT, ERR_INTERNAL = range(9)
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_STATE", 3: "OOM", 4: "CUDA", 5: "UNSUPPORTED", 6: "NUMERIC", 7: "TIMEOUT",
+                8: "INTERNAL"}
 LOSS = {"hinge": 0, "logistic": 1, "ridge": 2}
 FMT = {"dense": 0, "csr": 1, "csc": 2}
 MEM_HOST, MEM_DEVICE = 0, 1

@@ -96,6 +96,7 @@ chicle_status_t check_status(chicle_glm *h)
     const uint32_t bits = *h->h_status;
     if (bits == 0) return CHICLE_OK;
     (void)cudaMemsetAsync(h->d_status, 0, sizeof(uint32_t), h->stream);
+    if (bits & ST_BOUNDS) return fail(h, CHICLE_ERR_INTERNAL, "a bounds check of a CHICLE_DEBUG_BOUNDS build failed");
     if (bits & ST_WAIT_TIMEOUT) return fail(h, CHICLE_ERR_TIMEOUT, "a bounded wait inside a kernel ran out");
     if (bits & ST_BAD_INDEX) return fail(h, CHICLE_ERR_INVALID_ARG, "indptr not monotone or an index out of range");
     if (bits & ST_BAD_LABEL) return fail(h, CHICLE_ERR_INVALID_ARG, "labels must be +1 or -1 for hinge and logistic");

@@ -17,7 +17,19 @@ enum : uint32_t {
     ST_BAD_INDEX = 1u << 2,        // index outside [0, dim) or indptr not monotone
     ST_WAIT_TIMEOUT = 1u << 3,     // a bounded wait inside a kernel ran out
     ST_NONFINITE_STEP = 1u << 4,   // a coordinate step produced NaN/Inf
+    ST_BOUNDS = 1u << 5,           // a -DCHICLE_DEBUG_BOUNDS build: an index that a kernel loaded lay outside its array
 };
+
+// A -DCHICLE_DEBUG_BOUNDS build checks every index that the solvers and the gap kernels load from memory (visiting
+// order entries, row extents, entry ids, record directory entries, record sizes) before it is used as an address.
+// A failed check sets ST_BOUNDS in the status word and the access is skipped (the value is replaced by a harmless
+// one): never a trap, never an out-of-range access. The normal build compiles the checks away.
+#ifdef CHICLE_DEBUG_BOUNDS
+#define CHICLE_IN_BOUNDS(status, cond) ((cond) ? true : (atomicOr((status), (uint32_t)ST_BOUNDS), false))
+#else
+#define CHICLE_IN_BOUNDS(status, cond) true
+#endif
+
 
 // One SplitMix64 output for state x (published generator; a bijection on 64-bit words).
 __host__ __device__ __forceinline__ uint64_t mix64(uint64_t x)

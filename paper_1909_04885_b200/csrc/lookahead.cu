@@ -122,6 +122,7 @@ struct LookParams {
     int32_t hotc;                // entry ids per CTA kept in shared memory
     int64_t n_blocks;
     int64_t drop_block;          // test aid: this block's records are left unpublished (-1: none)
+    int64_t nnz;                 // entries of the matrix (what a coordinate's extent is checked against in a debug build)
     int32_t model_in;            // the round's first chain launch: row k of the update workspace holds U_k and is turned
                                  // into the local model w = v + sigma' U_k in place
     int32_t model_out;           // the round's last chain launch: the row is turned back into U_k. Between a round's
@@ -136,6 +137,21 @@ struct LookParams {
 #endif
 
 __device__ __forceinline__ int64_t steps_of(const LookParams &P, int64_t k, int64_t nk) { return partition_steps(P.S, k, nk); }
+// (debug build) an entry id as loaded from the matrix: id 0 stands in for one outside [0, dim) (the call then ends with
+// the bounds status, its arithmetic is of no interest; what matters is that nothing is addressed with the bad id)
+__device__ __forceinline__ int32_t checked_id(const LookParams &P, int32_t id)
+{
+    return CHICLE_IN_BOUNDS(P.S.status, id >= 0 && (int64_t)id < P.S.dim) ? id : 0;
+}
+// (debug build) a visiting-order entry and the extent of its coordinate: an empty coordinate 0 if either is off
+__device__ __forceinline__ void checked_extent(const LookParams &P, int32_t &c, int64_t &rs, int32_t &n)
+{
+    if (!CHICLE_IN_BOUNDS(P.S.status, c >= 0 && (int64_t)c < P.S.n_coord)) c = 0;
+    rs = P.S.indptr[c];
+    const int64_t len = P.S.indptr[c + 1] - rs;
+    n = (int32_t)len;
+    if (!CHICLE_IN_BOUNDS(P.S.status, rs >= 0 && len >= 0 && len <= 0x7fffffff && rs + len <= P.nnz)) { rs = 0; n = 0; }
+}
 __device__ __forceinline__ void block_to_part(const LookParams &P, int64_t bid, int &k, int64_t &b)
 {
     int32_t lo = 0, hi = P.K; // blk_base[lo] <= bid < blk_base[hi] (partitions may differ in size)
@@ -295,9 +311,8 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
         int64_t rs = 0;
         int32_t n = 0;
         if (lane < cnt) {
-            const int32_t c = P.S.perm[off + b * kLB + lane];
-            rs = P.S.indptr[c];
-            n = (int32_t)(P.S.indptr[c + 1] - rs);
+            int32_t c = P.S.perm[off + b * kLB + lane];
+            checked_extent(P, c, rs, n);
             hd = make_hdr<LOSS>(P.S, c);
         }
         sh.hdr[lane] = hd;
@@ -325,9 +340,8 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
         int64_t rs = 0;
         int32_t n = 0;
         if (lane < ncnt) {
-            const int32_t c = P.S.perm[off + (b + 1) * kLB + lane];
-            rs = P.S.indptr[c];
-            n = (int32_t)(P.S.indptr[c + 1] - rs);
+            int32_t c = P.S.perm[off + (b + 1) * kLB + lane];
+            checked_extent(P, c, rs, n);
             hd = make_hdr<LOSS>(P.S, c);
         }
         sh.nrs[lane] = rs;
@@ -371,7 +385,7 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int e = lane + 32 * c;
-                ids4[c] = e < n ? P.S.indices[rs + e] : -1;
+                ids4[c] = e < n ? checked_id(P, P.S.indices[rs + e]) : -1;
                 vals4[c] = e < n ? P.S.values[rs + e] : 0.0f;
             }
             auto take = [&](int e, int32_t id, float x) {
@@ -406,7 +420,7 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
                 if (32 * c < n) take(lane + 32 * c, ids4[c], vals4[c]);
             for (int e0 = 128; e0 < n; e0 += 32) {
                 const int e = e0 + lane;
-                take(e, e < n ? P.S.indices[rs + e] : -1, e < n ? P.S.values[rs + e] : 0.0f);
+                take(e, e < n ? checked_id(P, P.S.indices[rs + e]) : -1, e < n ? P.S.values[rs + e] : 0.0f);
             }
             if (lane == 0) {
 #pragma unroll
@@ -653,7 +667,7 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
 #pragma unroll
             for (int c = 0; c < 4; ++c) { // the first 128 entries are loaded before any is used
                 const int e = lane + 32 * c;
-                ids4[c] = e < n ? P.S.indices[rs + e] : -1;
+                ids4[c] = e < n ? checked_id(P, P.S.indices[rs + e]) : -1;
                 vals4[c] = e < n ? P.S.values[rs + e] : 0.0f;
             }
             auto take = [&](int32_t id, float x_l) {
@@ -693,7 +707,7 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
                 if (32 * c < n) take(ids4[c], vals4[c]);
             for (int e0 = 128; e0 < n; e0 += 32) {
                 const int e = e0 + lane;
-                take(e < n ? P.S.indices[rs + e] : -1, e < n ? P.S.values[rs + e] : 0.0f);
+                take(e < n ? checked_id(P, P.S.indices[rs + e]) : -1, e < n ? P.S.values[rs + e] : 0.0f);
             }
             __syncwarp();
             {
@@ -816,6 +830,7 @@ template <int LOSS> __device__ __forceinline__ void prepare_block_dense(const Lo
         const bool on = jj < (next ? ncnt : cnt);
         int32_t c = 0;
         if (on) c = P.S.perm[off + (b + (next ? 1 : 0)) * kLB + jj];
+        if (!CHICLE_IN_BOUNDS(P.S.status, c >= 0 && (int64_t)c < P.S.n_coord)) c = 0;
         const int64_t rs = (int64_t)c * dim;
         for (int e = lane; e < dim; e += 32) {
             const float x = on ? P.S.values[rs + e] : 0.0f;
@@ -1114,13 +1129,16 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                 const uint32_t w_base = smem_u32(W);
                 for (int j = 0; j < cnt; ++j) {
                     const CHdr h = H.hdr[j];
+                    if (!CHICLE_IN_BOUNDS(S.status, h.coord >= 0 && (int64_t)h.coord < S.n_coord)) continue;
                     const int64_t rs = DENSE ? (int64_t)h.coord * S.dim : S.indptr[h.coord];
-                    const int n = DENSE ? (int)S.dim : (int)(S.indptr[h.coord + 1] - rs);
+                    int n = DENSE ? (int)S.dim : (int)(S.indptr[h.coord + 1] - rs);
+                    if (!CHICLE_IN_BOUNDS(S.status, DENSE || (rs >= 0 && n >= 0 && rs + n <= P.nnz))) n = 0;
                     const int32_t *ix = S.indices + rs;
                     const float *xv = S.values + rs;
                     float acc = 0.0f, delta, new_state;
                     for (int e = lane; e < n; e += 32) {
-                        const uint32_t g = DENSE ? (uint32_t)e : (uint32_t)ix[e];
+                        uint32_t g = DENSE ? (uint32_t)e : (uint32_t)ix[e];
+                        if (!CHICLE_IN_BOUNDS(S.status, (int64_t)g < S.dim)) g = 0u;
                         const float ww = g < hot_total ? ld_cluster_f32(mapa_u32(w_base + 4u * (g >> logC), g & (uint32_t)(C - 1)))
                                                        : __ldcg(Uk + g);
                         acc = fmaf(xv[e], ww, acc);
@@ -1134,7 +1152,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                     }
                     if (delta != 0.0f)
                         for (int e = lane; e < n; e += 32) {
-                            const uint32_t g = DENSE ? (uint32_t)e : (uint32_t)ix[e];
+                            uint32_t g = DENSE ? (uint32_t)e : (uint32_t)ix[e];
+                            if (!CHICLE_IN_BOUNDS(S.status, (int64_t)g < S.dim)) continue;
                             if (g < hot_total) {
                                 const uint32_t a = mapa_u32(w_base + 4u * (g >> logC), g & (uint32_t)(C - 1));
                                 st_cluster_f32(a, fmaf(sigma * delta, xv[e], ld_cluster_f32(a)));
@@ -1235,7 +1254,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                             my_delta = 0.0f;
                             my_state = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? hp1[i] : hp3[i] * hp1[i];
                         }
-                        S.alpha[hcoord[i]] = my_state; // (the four copies of a lane store the same value)
+                        if (CHICLE_IN_BOUNDS(S.status, hcoord[i] >= 0 && (int64_t)hcoord[i] < S.n_coord))
+                            S.alpha[hcoord[i]] = my_state; // (the four copies of a lane store the same value)
                     }
                     dl[i] = my_delta;
                 }
@@ -1278,7 +1298,9 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
             const uint32_t bar = smem_u32(&ctl.subfull[blk & (kSubSlots - 1)]);
             // (the slot is only ever written by the copy engine and read by loads that are done by now)
             const unsigned long long offset = ((unsigned long long)d[1] << 32) | d[0];
-            const uint32_t bytes = d[2] <= L.sub_stride ? d[2] : 0u;
+            uint32_t bytes = d[2] <= L.sub_stride ? d[2] : 0u;
+            if (!CHICLE_IN_BOUNDS(S.status, (offset & 15ull) == 0ull && offset + bytes <= P.pool_off + P.pool_cap))
+                bytes = 0u; // (an entry that points outside the region: as if no record had been written)
             const bool mine = blk < nb && wt == 0;
             if (mine && bytes == 0) {
                 // no record: nothing will arrive, say so now
@@ -1317,6 +1339,13 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
             LA_T(wg0);
             const unsigned char *rec = sub_at(x);
             const SubHead &h = *reinterpret_cast<const SubHead *>(rec);
+            // (debug build) a record whose sizes do not fit its slot is not read: as if its wait had run out
+            if (!CHICLE_IN_BOUNDS(S.status, h.cnt >= 0 && h.cnt <= kLB &&
+                                                (DENSE || (h.n >= 0 && h.n <= P.nzcap && h.T >= 0 && h.T <= P.nzcap / 2 && h.roff[kLB] == h.n)))) {
+                failed = true;
+                ++fg;
+                return !DENSE;
+            }
             const float *val = reinterpret_cast<const float *>(rec + sizeof(SubHead));
             const uint32_t slot = (uint32_t)(fg & 1);
             if (DENSE) {
@@ -1353,7 +1382,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                             const bool on = e < hi;
                             x8[u] = on ? val[e] : 0.0f;
                             const uint32_t g = on ? (meta[e] & kIdMask) : 0u;
-                            u8[u] = ldcg_if(Uk + g, on);
+                            u8[u] = ldcg_if(Uk + g, on && CHICLE_IN_BOUNDS(S.status, (int64_t)g < S.dim));
                         }
 #pragma unroll
                         for (int u = 0; u < 8; ++u) acc = fmaf(x8[u], u8[u], acc);
@@ -1373,8 +1402,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                         const bool on = e < hi;
                         x[u] = on ? val[e] : 0.0f;
                         const uint32_t g = on ? (meta[e] & kIdMask) : 0u;
-                        cold[u] = on && g >= hot_total;
-                        hv[u] = W[cold[u] ? 0u : (g >> logC)];
+                        cold[u] = on && g >= hot_total && CHICLE_IN_BOUNDS(S.status, (int64_t)g < S.dim);
+                        hv[u] = W[g < hot_total ? (g >> logC) : 0u];
                         uu[u] = ldcg_if(Uk + (cold[u] ? g : 0u), cold[u]);
                     }
                     float acc = x[0] * (cold[0] ? uu[0] : hv[0]);
@@ -1390,8 +1419,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                             const bool on = e < hi;
                             x4[u] = on ? val[e] : 0.0f;
                             const uint32_t g = on ? (meta[e] & kIdMask) : 0u;
-                            c4[u] = on && g >= hot_total;
-                            h4[u] = W[c4[u] ? 0u : (g >> logC)];
+                            c4[u] = on && g >= hot_total && CHICLE_IN_BOUNDS(S.status, (int64_t)g < S.dim);
+                            h4[u] = W[g < hot_total ? (g >> logC) : 0u];
                             u4[u] = ldcg_if(Uk + (c4[u] ? g : 0u), c4[u]);
                         }
 #pragma unroll
@@ -1476,9 +1505,10 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                             }
 #pragma unroll
                             for (int u = 0; u < 8; ++u) {
-                                const bool shared_id = (m8[u] >> 31) != 0u;
+                                const bool shared_id = (m8[u] >> 31) != 0u && CHICLE_IN_BOUNDS(S.status, c8[u] < P.nzcap);
                                 sts_f32(shared_id ? a_prod + 4u * (uint32_t)c8[u] : a_sink, p8[u]);
-                                const bool far = !shared_id && p8[u] != 0.0f; // (beyond the coordinate's end p8 is 0)
+                                const bool far = (m8[u] >> 31) == 0u && p8[u] != 0.0f && // (beyond the coordinate's end p8 is 0)
+                                                 CHICLE_IN_BOUNDS(S.status, (int64_t)(m8[u] & kIdMask) < S.dim);
                                 red_add_if(Uk + (far ? (m8[u] & kIdMask) : 0u), sigma * p8[u], far);
                             }
                         }
@@ -1508,18 +1538,20 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                         for (int u = 0; u < 2; ++u) {
                             const uint32_t g = m[u] & kIdMask;
                             const bool shared_id = (m[u] >> 31) != 0u, hot = g < hot_total;
-                            const uint32_t addr = !on[u] ? a_sink : (shared_id ? a_prod + 4u * (uint32_t)cp[u] : (hot ? a_w + 4u * (g >> logC) : a_sink));
+                            const bool list_ok = CHICLE_IN_BOUNDS(S.status, !shared_id || cp[u] < P.nzcap);
+                            const uint32_t addr = (!on[u] || !list_ok) ? a_sink : (shared_id ? a_prod + 4u * (uint32_t)cp[u] : (hot ? a_w + 4u * (g >> logC) : a_sink));
                             sts_f32(addr, shared_id ? p[u] : fmaf(sigma, p[u], w2[u]));
-                            const bool far = on[u] && !shared_id && !hot && p[u] != 0.0f;
+                            const bool far = on[u] && !shared_id && !hot && p[u] != 0.0f && CHICLE_IN_BOUNDS(S.status, (int64_t)g < S.dim);
                             red_add_if(Uk + (far ? g : 0u), sigma * p[u], far); // a reduction at L2, nothing waits for it
                         }
                         for (int e = lo + 16; e < hi; e += 8) {
                             const uint32_t mm = meta[e];
                             const uint32_t g = mm & kIdMask;
                             const float pp = d * val[e];
-                            if (mm & 0x80000000u) prod[cpos[e]] = pp;
-                            else if (g < hot_total) W[g >> logC] = fmaf(sigma, pp, W[g >> logC]);
-                            else if (pp != 0.0f) atomicAdd(Uk + g, sigma * pp);
+                            if (mm & 0x80000000u) {
+                                if (CHICLE_IN_BOUNDS(S.status, cpos[e] < P.nzcap)) prod[cpos[e]] = pp;
+                            } else if (g < hot_total) W[g >> logC] = fmaf(sigma, pp, W[g >> logC]);
+                            else if (pp != 0.0f && CHICLE_IN_BOUNDS(S.status, (int64_t)g < S.dim)) atomicAdd(Uk + g, sigma * pp);
                         }
                     }
                     work_bar();
@@ -1541,6 +1573,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_lookahead_chain(const Look
                             o0[u] = on[u] ? offs[t] + quarter : 0;
                             o1[u] = on[u] ? offs[t + 1] : 0;
                             g3[u] = on[u] ? ids[t] : 0u;
+                            if (!CHICLE_IN_BOUNDS(S.status, o1[u] <= P.nzcap && (int64_t)g3[u] < S.dim)) { o1[u] = 0; on[u] = false; }
                         }
                         float vv[2][8];
 #pragma unroll
@@ -1979,6 +2012,7 @@ cudaError_t launch_lookahead_solver(Glm &g, const SolverParams &S)
         p.hotc = g.la_hotc;
         p.n_blocks = blocks[(size_t)s];
         p.drop_block = (drop && s == 0) ? atoll(drop) : -1;
+        p.nnz = g.nnz;
         p.model_in = s == 0 ? 1 : 0;
         p.model_out = s == Sn - 1 ? 1 : 0;
     }

@@ -218,7 +218,7 @@ __global__ void __launch_bounds__(kThreads)
 k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices,
                const float *__restrict__ values, const float *__restrict__ labels, const float *__restrict__ state,
                const float *__restrict__ vec /* the shared vector */, const float *__restrict__ v,
-               int64_t n_coord, int64_t dim, double lam_n, double *__restrict__ partials)
+               int64_t n_coord, int64_t dim, double lam_n, double *__restrict__ partials, uint32_t *status)
 {
     __shared__ double sh[kThreads][2];
     __shared__ double sh2[kWarpsPerBlock][2];
@@ -272,6 +272,7 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
                     if (e < re[r]) {
                         ix[r][ch] = indices[e];
                         xv[r][ch] = values[e];
+                        if (!CHICLE_IN_BOUNDS(status, ix[r][ch] >= 0 && (int64_t)ix[r][ch] < dim)) ix[r][ch] = -1;
                     }
                 }
             double dot[kGapRows];
@@ -287,6 +288,7 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
                     }
                 for (int64_t e = rs[r] + 32 * kGapChunks + lane; e < re[r]; e += 32) { // the rest of a long coordinate
                     const int32_t i = indices[e];
+                    if (!CHICLE_IN_BOUNDS(status, i >= 0 && (int64_t)i < dim)) continue;
                     double t = (double)vec[i];
                     if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) t -= (double)labels[i];
                     dot[r] = fma((double)values[e], t, dot[r]);
@@ -543,6 +545,7 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
                     }
 #pragma unroll
                     for (int q = 0; q < kMaxPer; ++q) {
+                        if (!CHICLE_IN_BOUNDS(status, ii[q] >= 0 && (int64_t)ii[q] < dim)) ii[q] = 0;
                         const bool far = ii[q] >= hot_n;
                         hh[q] = sm.vhot[far ? 0 : ii[q]];
                         tt[q] = gap_ldg_if(vec + (far ? ii[q] : 0), far);
@@ -557,7 +560,8 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
                 }
             } else {
                 for (int64_t e = rs + sub; e < re; e += TPR) {
-                    const int32_t i = indices[e];
+                    int32_t i = indices[e];
+                    if (!CHICLE_IN_BOUNDS(status, i >= 0 && (int64_t)i < dim)) i = 0;
                     float t;
                     if (i < hot_n) t = sm.vhot[i];
                     else t = vec[i] - (LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? labels[i] : 0.0f);
@@ -781,7 +785,7 @@ template <int LOSS> cudaError_t launch_gap_loss(Glm &g)
         if (e != cudaSuccess) return e;
     } else {
         k_gap_partials<LOSS><<<nb, kThreads, 0, g.stream>>>(g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.v, g.n_coord,
-                                                            g.dim, lam_n, g.gap_partials);
+                                                            g.dim, lam_n, g.gap_partials, g.d_status);
     }
     k_gap_final<LOSS><<<1, 128, 0, g.stream>>>(g.gap_partials, nb, n, (double)g.lambda, g.gap_out);
     return cudaGetLastError();
