@@ -431,6 +431,7 @@ template <int LOSS, int R, int PER>
 __global__ void __launch_bounds__(kGapConsumers + 32, 1)
 k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices, const float *__restrict__ values,
              const float *__restrict__ labels, const float *__restrict__ state, const float *__restrict__ vec,
+             const float *__restrict__ gvec /* what the dot products gather from: v, or for ridge the residual v - y */,
              int64_t n_coord, int64_t dim, double lam_n, double *__restrict__ partials, uint32_t *status)
 {
     constexpr int TPR = kGapConsumers / R; // threads per coordinate
@@ -450,7 +451,7 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
     }
     const int hot_n = (int)(dim < kGapHot ? dim : kGapHot);
     for (int i = tid; i < hot_n; i += kGapConsumers + 32)
-        sm.vhot[i] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? vec[i] - labels[i] : vec[i];
+        sm.vhot[i] = gvec[i];
     __syncthreads();
     const int64_t ntiles = (n_coord + R - 1) / R;
     const int64_t first = blockIdx.x, step = gridDim.x;
@@ -533,7 +534,7 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
                 const uint32_t a_idx = smem_u32(&sm.idx[st][0]), a_val = smem_u32(&sm.val[st][0]);
                 for (int e0 = (int)(rs - base) + sub; e0 < hi; e0 += TPR * kMaxPer) {
                     int32_t ii[kMaxPer];
-                    float xx[kMaxPer], tt[kMaxPer], yy[kMaxPer], hh[kMaxPer];
+                    float xx[kMaxPer], tt[kMaxPer], hh[kMaxPer];
 #pragma unroll
                     for (int q = 0; q < kMaxPer; ++q) {
                         const int e = e0 + q * TPR;
@@ -548,14 +549,12 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
                         if (!CHICLE_IN_BOUNDS(status, ii[q] >= 0 && (int64_t)ii[q] < dim)) ii[q] = 0;
                         const bool far = ii[q] >= hot_n;
                         hh[q] = sm.vhot[far ? 0 : ii[q]];
-                        tt[q] = gap_ldg_if(vec + (far ? ii[q] : 0), far);
-                        yy[q] = LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? gap_ldg_if(labels + (far ? ii[q] : 0), far) : 0.0f;
+                        tt[q] = gap_ldg_if(gvec + (far ? ii[q] : 0), far);
                     }
 #pragma unroll
                     for (int q = 0; q < kMaxPer; ++q) {
-                        // (x is 0 beyond the coordinate's end; fp32 v - y for the staged head, as the solvers' residual)
-                        if (LOSS == CHICLE_LOSS_RIDGE_PRIMAL) dot = fmaf(xx[q], ii[q] >= hot_n ? tt[q] - yy[q] : hh[q], dot);
-                        else dot = fmaf(xx[q], ii[q] >= hot_n ? tt[q] : hh[q], dot);
+                        // (x is 0 beyond the coordinate's end)
+                        dot = fmaf(xx[q], ii[q] >= hot_n ? tt[q] : hh[q], dot);
                     }
                 }
             } else {
@@ -564,7 +563,7 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
                     if (!CHICLE_IN_BOUNDS(status, i >= 0 && (int64_t)i < dim)) i = 0;
                     float t;
                     if (i < hot_n) t = sm.vhot[i];
-                    else t = vec[i] - (LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? labels[i] : 0.0f);
+                    else t = gvec[i];
                     dot = fmaf(values[e], t, dot);
                 }
             }
@@ -753,7 +752,8 @@ template <int LOSS, int R, int PER> cudaError_t launch_gap_stream_per(Glm &g, in
     auto kern = k_gap_stream<LOSS, R, PER>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(GapShared));
     if (e != cudaSuccess) return e;
-    kern<<<nb, kGapConsumers + 32, sizeof(GapShared), g.stream>>>(g.indptr, g.indices, g.values, g.labels, g.alpha, g.v, g.n_coord,
+    kern<<<nb, kGapConsumers + 32, sizeof(GapShared), g.stream>>>(g.indptr, g.indices, g.values, g.labels, g.alpha, g.v,
+                                                                   LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? g.resid : g.v, g.n_coord,
                                                                    g.dim, lam_n, g.gap_partials, g.d_status);
     return cudaGetLastError();
 }
@@ -772,8 +772,8 @@ template <int LOSS> cudaError_t launch_gap_loss(Glm &g)
     const double lam_n = (double)g.lambda * n;
     int nb = g.gap_blocks;
     const char *force = getenv("CHICLE_FORCE_VARIANT"); // debugging aid: "gapwarp" selects the warp-per-coordinate kernel
-    if (g.indptr && g.hot_variant && !(force && strcmp(force, "gapwarp") == 0)) {
-        // skewed ids: the streamed kernel, one block per SM; coordinates per tile: as many as keep a tile's non-zeros
+    if (g.indptr && !(force && strcmp(force, "gapwarp") == 0)) {
+        // sparse data: the streamed kernel, one block per SM; coordinates per tile: as many as keep a tile's non-zeros
         // comfortably inside a stage
         nb = g.sm_count < g.gap_blocks ? g.sm_count : g.gap_blocks;
         const double avg = (double)g.nnz / (double)g.n_coord;

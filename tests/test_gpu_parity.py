@@ -419,6 +419,13 @@ def test_ids_beyond_the_shared_memory_part_across_slices(cluster, monkeypatch):
     run_parity(datagen.make("hinge_csr", 4 if cluster == "1" else 2), rounds=2)
 
 
+def test_warp_per_coordinate_gap_kernel_on_sparse_data(monkeypatch):
+    # sparse data take the streamed gap kernel by default; the warp-per-coordinate kernel stays selectable
+    monkeypatch.setenv("CHICLE_FORCE_VARIANT", "gapwarp")
+    run_parity(datagen.make("hinge_csr", 100), rounds=2)
+    run_parity(datagen.make("ridge_csc", 100), rounds=2)
+
+
 def test_a_missing_record_ends_in_a_timeout_status_and_the_handle_stays_usable(monkeypatch):
     # Failure detection without a fault: one block's records are left unpublished (a host-side test aid), so the chain
     # kernel finds nothing to copy, sets the status word with no copy in flight, every wait in the cluster runs out
