@@ -373,7 +373,7 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
 }
 
 // Sparse formats, streamed: the coordinates of a block's tile lie one after the other in memory, so their indices and
-// values are two contiguous ranges, which a producer warp brings into a three-stage shared-memory ring with bulk
+// values are two contiguous ranges, which a producer warp brings into a shared-memory ring of two or three stages with bulk
 // copies (16-byte aligned windows; the bytes in flight no longer depend on registers or on how many warps fit). The
 // sixteen consumer warps take R coordinates per tile, 512 / R threads each (every thread a fixed subset of the
 // coordinate's entries, all gathers from the shared vector issued before the first use), and add the partial dot
@@ -383,10 +383,13 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
 // vector in its shared memory (ids are frequency-ranked: they take most of the gathers); the kernel is used when the
 // ids are skewed, one block per SM. Every wait is bounded; when one runs out the status word says so and all roles
 // leave.
-constexpr int kGapStages = 3;
-constexpr int kGapHot = 32768;             // entries of the shared vector staged per block (128 KB)
-constexpr int kGapCapNz = 3584;            // non-zeros a stage holds
-constexpr int kGapStageElems = kGapCapNz + 8; // + the window's alignment slack
+// Two shapes of the shared memory: 32 768 staged entries of the shared vector (128 KB) with stages of 3 584 non-zeros,
+// or 22 528 entries (88 KB) with stages of 5 248: the larger stages hold tiles of 128 short coordinates, which halves
+// the per-tile work (waits, extents, the fp64 gap terms) per non-zero.
+constexpr int kGapHot = 32768, kGapCapNz = 3584;
+constexpr int kGapHotWide = 22528, kGapCapNzWide = 5248;
+// (A two-stage ring of still larger stages for coordinates of about 50 entries was slower: 0.184 against 0.167 ms at
+// 1 M coordinates.)
 constexpr int kGapConsumers = 512;
 
 // Bounded wait without back-off (try_wait itself parks the thread for a while): every lane calls it, lane 0 polls.
@@ -415,19 +418,20 @@ __device__ __forceinline__ float gap_ldg_if(const float *p, bool on)
     return v;
 }
 
-struct GapShared {
-    alignas(16) float vhot[kGapHot];       // the head of the shared vector (ridge: of v - y)
-    alignas(16) int32_t idx[kGapStages][kGapStageElems];
-    alignas(16) float val[kGapStages][kGapStageElems];
-    alignas(8) uint64_t full[kGapStages];  // the stage's copies have landed (or the tile was marked as not staged)
-    alignas(8) uint64_t empty[kGapStages]; // the consumer warps have finished with the stage
-    long long base[kGapStages];            // first element of the stage's window in the global arrays; -1: not staged
+template <int HOT, int CAP, int STAGES> struct GapShared {
+    static constexpr int kStageElems = CAP + 8; // + the window's alignment slack
+    alignas(16) float vhot[HOT];           // the head of the shared vector (ridge: of v - y)
+    alignas(16) int32_t idx[STAGES][kStageElems];
+    alignas(16) float val[STAGES][kStageElems];
+    alignas(8) uint64_t full[STAGES];  // the stage's copies have landed (or the tile was marked as not staged)
+    alignas(8) uint64_t empty[STAGES]; // the consumer warps have finished with the stage
+    long long base[STAGES];            // first element of the stage's window in the global arrays; -1: not staged
     double sh[kGapConsumers][2];
     double sh2[kGapConsumers / 32][2];
     int abort_flag;
 };
 
-template <int LOSS, int R, int PER>
+template <int LOSS, int R, int PER, int HOT, int CAP, int STAGES>
 __global__ void __launch_bounds__(kGapConsumers + 32, 1)
 k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices, const float *__restrict__ values,
              const float *__restrict__ labels, const float *__restrict__ state, const float *__restrict__ vec,
@@ -437,7 +441,9 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
     constexpr int TPR = kGapConsumers / R; // threads per coordinate
     constexpr int kMaxPer = PER;           // entries a thread keeps in flight (6 or 8: the fewer idle slots, the fewer instructions)
     extern __shared__ __align__(128) unsigned char gap_smem[];
-    GapShared &sm = *reinterpret_cast<GapShared *>(gap_smem);
+    using Shared = GapShared<HOT, CAP, STAGES>;
+    constexpr int kGapStages = STAGES;
+    Shared &sm = *reinterpret_cast<Shared *>(gap_smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const double inv_lam_n = 1.0 / lam_n;
     volatile int *abort_flag = &sm.abort_flag;
@@ -449,7 +455,7 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    const int hot_n = (int)(dim < kGapHot ? dim : kGapHot);
+    const int hot_n = (int)(dim < HOT ? dim : HOT);
     for (int i = tid; i < hot_n; i += kGapConsumers + 32)
         sm.vhot[i] = gvec[i];
     __syncthreads();
@@ -482,7 +488,7 @@ k_gap_stream(const int64_t *__restrict__ indptr, const int32_t *__restrict__ ind
                 const uint32_t bar = smem_u32(&sm.full[st]);
                 // the stage was read by ordinary loads: order them before the copy engine's writes
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                if (elems > 0 && elems <= kGapStageElems) {
+                if (elems > 0 && elems <= Shared::kStageElems) {
                     sm.base[st] = w0;
                     const uint32_t bytes = (uint32_t)elems * 4u;
                     mbar_arrive_expect_tx(bar, 2u * bytes);
@@ -747,12 +753,14 @@ cudaError_t launch_refresh_resid(Glm &g)
     return cudaGetLastError();
 }
 
-template <int LOSS, int R, int PER> cudaError_t launch_gap_stream_per(Glm &g, int nb, double lam_n)
+template <int LOSS, int R, int PER, int HOT = kGapHot, int CAP = kGapCapNz, int STAGES = 3>
+cudaError_t launch_gap_stream_per(Glm &g, int nb, double lam_n)
 {
-    auto kern = k_gap_stream<LOSS, R, PER>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(GapShared));
+    using Shared = GapShared<HOT, CAP, STAGES>;
+    auto kern = k_gap_stream<LOSS, R, PER, HOT, CAP, STAGES>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Shared));
     if (e != cudaSuccess) return e;
-    kern<<<nb, kGapConsumers + 32, sizeof(GapShared), g.stream>>>(g.indptr, g.indices, g.values, g.labels, g.alpha, g.v,
+    kern<<<nb, kGapConsumers + 32, sizeof(Shared), g.stream>>>(g.indptr, g.indices, g.values, g.labels, g.alpha, g.v,
                                                                    LOSS == CHICLE_LOSS_RIDGE_PRIMAL ? g.resid : g.v, g.n_coord,
                                                                    g.dim, lam_n, g.gap_partials, g.d_status);
     return cudaGetLastError();
@@ -779,6 +787,8 @@ template <int LOSS> cudaError_t launch_gap_loss(Glm &g)
         const double avg = (double)g.nnz / (double)g.n_coord;
         cudaError_t e;
         if (avg * 128 <= 3300) e = launch_gap_stream<LOSS, 128>(g, nb, lam_n);
+        else if (avg <= 39.5 && avg * 128 * 1.05 <= kGapCapNzWide) // (four threads per coordinate, ten entries each)
+            e = launch_gap_stream_per<LOSS, 128, 10, kGapHotWide, kGapCapNzWide>(g, nb, lam_n);
         else if (avg * 64 <= 3300) e = launch_gap_stream<LOSS, 64>(g, nb, lam_n);
         else if (avg * 32 <= 3300) e = launch_gap_stream<LOSS, 32>(g, nb, lam_n);
         else e = launch_gap_stream<LOSS, 16>(g, nb, lam_n);
