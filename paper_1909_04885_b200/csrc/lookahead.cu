@@ -374,6 +374,20 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
     if (!slow) {
         // ---- the block's non-zeros into shared memory, every id into the table; how many fall to each CTA. The
         //      first 128 entries of a coordinate are loaded before any is used.
+        //      The loads of a warp's next coordinate are issued before this one's entries are inserted.
+        int32_t ids_nx[4];
+        float vals_nx[4];
+        auto load4 = [&](int j, int32_t (&ids)[4], float (&vals)[4]) {
+            const int n = j < cnt ? sh.nnz[j] : 0;
+            const int64_t rs = j < cnt ? sh.rs[j] : 0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int e = lane + 32 * c;
+                ids[c] = e < n ? checked_id(P, P.S.indices[rs + e]) : -1;
+                vals[c] = e < n ? P.S.values[rs + e] : 0.0f;
+            }
+        };
+        load4(warp, ids_nx, vals_nx);
         for (int j = warp; j < cnt; j += NW) {
             const int n = sh.nnz[j], r0 = sh.roff[j];
             const int64_t rs = sh.rs[j];
@@ -383,11 +397,8 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
             int32_t ids4[4];
             float vals4[4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const int e = lane + 32 * c;
-                ids4[c] = e < n ? checked_id(P, P.S.indices[rs + e]) : -1;
-                vals4[c] = e < n ? P.S.values[rs + e] : 0.0f;
-            }
+            for (int c = 0; c < 4; ++c) { ids4[c] = ids_nx[c]; vals4[c] = vals_nx[c]; }
+            load4(j + NW, ids_nx, vals_nx);
             auto take = [&](int e, int32_t id, float x) {
                 const bool on = id >= 0;
                 if (on) {
