@@ -664,8 +664,28 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
     PRE_T(6);
     // ---- cross Gram matrix with the next block: a warp per coordinate j of the next block, whose non-zeros come
     //      straight from the matrix and are looked up in this block's table; lane l collects x_j . x_l
+    //      (the first 128 entries of a warp's next coordinate are loaded while it works on the current one)
+    int32_t xids_nx[4];
+    float xvals_nx[4];
+    auto xload4 = [&](int j, int32_t (&ids)[4], float (&vals)[4]) {
+        const bool have = carry && j < sh.ncnt;
+        const int n = have ? sh.nnnz[j] : 0;
+        const int64_t rs = have ? sh.nrs[j] : 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int e = lane + 32 * c;
+            ids[c] = e < n ? checked_id(P, P.S.indices[rs + e]) : -1;
+            vals[c] = e < n ? P.S.values[rs + e] : 0.0f;
+        }
+    };
+    xload4(warp, xids_nx, xvals_nx);
     for (int j = warp; j < kLB; j += NW) {
         float acc = 0.0f;
+        int32_t ids4[4];
+        float vals4[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) { ids4[c] = xids_nx[c]; vals4[c] = xvals_nx[c]; }
+        xload4(j + NW, xids_nx, xvals_nx);
         if (carry && j < sh.ncnt) {
             const int n = sh.nnnz[j];
             const int64_t rs = sh.nrs[j];
@@ -673,14 +693,6 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
             int per_class[kMaxC];
 #pragma unroll
             for (int c = 0; c < kMaxC; ++c) per_class[c] = 0;
-            int32_t ids4[4];
-            float vals4[4];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) { // the first 128 entries are loaded before any is used
-                const int e = lane + 32 * c;
-                ids4[c] = e < n ? checked_id(P, P.S.indices[rs + e]) : -1;
-                vals4[c] = e < n ? P.S.values[rs + e] : 0.0f;
-            }
             auto take = [&](int32_t id, float x_l) {
                 uint32_t m_l = 0u;
                 int so_l = 0;
