@@ -238,9 +238,14 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
         e = cudaMemcpy2DAsync(h->values, (size_t)h->dim * 4, X->values, (size_t)X->ld * 4, (size_t)h->dim * 4,
                               (size_t)h->n_coord, kind, s);
     } else {
-        e = copy_in(h->values, X->values, nvals * 4, X->space, s);
-        if (e == cudaSuccess) e = copy_in(h->indptr, X->indptr, ((size_t)h->n_coord + 1) * 8, X->space, s);
+        // The structure first: its checks and the ranking of the ids need no values, so the values (half of the
+        // bytes) travel on the side stream, behind the indices, while those kernels run.
+        e = copy_in(h->indptr, X->indptr, ((size_t)h->n_coord + 1) * 8, X->space, s);
         if (e == cudaSuccess && nvals) e = copy_in(h->indices, X->indices, nvals * 4, X->space, s);
+        if (e == cudaSuccess) e = cudaEventRecord(h->la_ev_prep[0], s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->la_stream, h->la_ev_prep[0], 0);
+        if (e == cudaSuccess) e = copy_in(h->values, X->values, nvals * 4, X->space, h->la_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(h->la_ev_done[0], h->la_stream);
     }
     if (e == cudaSuccess) e = copy_in(h->labels, labels, (size_t)h->n_examples * 4, X->space, s);
     if (e == cudaSuccess) e = cudaMemsetAsync(h->alpha, 0, (size_t)h->n_coord * 4, s);
@@ -257,7 +262,7 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
         if (e != cudaSuccess) return bail_cuda(e, "reading indptr");
         if (ends[0] != 0 || ends[1] != h->nnz) return bail(CHICLE_ERR_INVALID_ARG, "indptr[0] != 0 or indptr[last] != nnz");
     }
-    e = launch_validate(*h);
+    e = launch_validate(*h, dense, true); // (sparse: the values are checked once they have arrived, below)
     if (e != cudaSuccess) return bail_cuda(e, "validation kernels");
     chicle_status_t st = check_status(h);
     if (st != CHICLE_OK) {
@@ -301,6 +306,16 @@ chicle_status_t chicle_glm_create(const chicle_matrix_t *X, const float *labels,
         if (force && strcmp(force, "flat") == 0) h->hot_variant = 0;
         if (force && strcmp(force, "hot") == 0) h->hot_variant = 1;
         if (force && strcmp(force, "hot128") == 0) h->hot_variant = 2;
+    }
+    if (!dense) {
+        e = cudaStreamWaitEvent(s, h->la_ev_done[0], 0);
+        if (e == cudaSuccess) e = launch_validate(*h, true, false);
+        if (e != cudaSuccess) return bail_cuda(e, "validation kernels");
+        st = check_status(h);
+        if (st != CHICLE_OK) {
+            const std::string msg = h->err;
+            return bail(st, msg);
+        }
     }
     e = launch_sqnorm(*h);
     if (e == cudaSuccess) e = launch_refresh_resid(*h);

@@ -148,7 +148,7 @@ struct Glm {
 };
 
 // ---- kernels' host launchers (each returns the launch error, work is enqueued on g.stream) -----------------
-cudaError_t launch_validate(Glm &g);
+cudaError_t launch_validate(Glm &g, bool values = true, bool rest = true); // the values array; labels and structure
 cudaError_t launch_sqnorm(Glm &g);
 cudaError_t launch_partition(Glm &g, int32_t K, uint64_t seed);           // fills owner, members
 cudaError_t launch_partition_chunks(Glm &g, int32_t K, int64_t C, const int64_t *chunk_off, const int32_t *chunk_task); // device arrays

@@ -682,11 +682,12 @@ k_shared_vector(const int64_t *__restrict__ indptr, const int32_t *__restrict__ 
 
 } // namespace
 
-cudaError_t launch_validate(Glm &g)
+cudaError_t launch_validate(Glm &g, bool values, bool rest)
 {
     const int64_t nvals = g.indptr ? g.nnz : g.n_coord * g.dim;
     const unsigned grid = (unsigned)g.sm_count * 8;
-    k_validate_values<<<grid, kThreads, 0, g.stream>>>(g.values, nvals, g.d_status);
+    if (values) k_validate_values<<<grid, kThreads, 0, g.stream>>>(g.values, nvals, g.d_status);
+    if (!rest) return cudaGetLastError();
     k_validate_labels<<<grid, kThreads, 0, g.stream>>>(g.labels, g.n_examples,
                                                        g.loss != CHICLE_LOSS_RIDGE_PRIMAL, g.d_status);
     if (g.indptr)
