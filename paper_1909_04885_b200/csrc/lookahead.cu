@@ -20,7 +20,9 @@
 //                         bits every run.
 //   k_lookahead_chain     one cluster of C CTAs per partition. Entry ids below C * HOT (ids are frequency-ranked)
 //                         live in shared memory for the whole kernel as w = v + sigma' U_k, id i in CTA i mod C;
-//                         the others are read from and added to row k of the update workspace in global memory.
+//                         the others live in row k of the update workspace in global memory, which holds the model
+//                         itself between the launches of a round (the first launch turns U_k into w in place, the
+//                         last one turns it back): one gather or one reduction per non-zero.
 //                         Warp 0 of CTA 0 runs the recurrence. The worker warps of every CTA loop over
 //                         "wait for block b's deltas, apply them to my part of the model, take my part of block
 //                         b + 2's dot products, send the 32 partial sums to CTA 0". Deltas and partial sums travel
