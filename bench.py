@@ -462,6 +462,10 @@ def run_b200(args):
             "roofline": {"bound": "hbm", "kernel": "k_lookahead_chain at %s (local SCD solvers: one thread-block cluster per partition)" % dom_key,
                          "achieved": dom["hbm_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dom["hbm_frac"],
                          "peak_kind": "of " + peak_kind, "traffic": traffic, "traffic_note": prof.get("traffic_note"),
+                         "traffic_detail": None if traffic is None else {
+                             "bytes": traffic, "captured_at_scale": 16, "extrapolated": True,
+                             "covers": "all chain launches of one round (19 at full size); bytes per coordinate step "
+                                       "from the ncu capture at 1/16 size times the steps of a round"},
                          "algorithmic_bytes_per_launch": H["algorithmic_bytes_per_round"],
                          "note": "a partition is walked strictly in order: K dependent chains and the throughput of the "
                                  "prepare kernel bound the local solvers, not HBM; achieved = algorithmic bytes of a round / time "
