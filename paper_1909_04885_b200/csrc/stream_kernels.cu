@@ -388,8 +388,10 @@ k_gap_partials(const int64_t *__restrict__ indptr, const int32_t *__restrict__ i
 // the per-tile work (waits, extents, the fp64 gap terms) per non-zero.
 constexpr int kGapHot = 32768, kGapCapNz = 3584;
 constexpr int kGapHotWide = 22528, kGapCapNzWide = 5248;
-// (A two-stage ring of still larger stages for coordinates of about 50 entries was slower: 0.184 against 0.167 ms at
-// 1 M coordinates.)
+// ... or 14 336 entries (56 KB) with stages of 6 912, for tiles of 128 coordinates of about 50 entries: 0.149 against
+// 0.161 ms per call at 1 M coordinates, although fewer gathers find their entry staged. (A two-stage ring with a larger
+// head was slower: 0.184 ms.)
+constexpr int kGapHotWider = 14336, kGapCapNzWider = 6912;
 constexpr int kGapConsumers = 512;
 
 // Bounded wait without back-off (try_wait itself parks the thread for a while): every lane calls it, lane 0 polls.
@@ -790,6 +792,8 @@ template <int LOSS> cudaError_t launch_gap_loss(Glm &g)
         if (avg * 128 <= 3300) e = launch_gap_stream<LOSS, 128>(g, nb, lam_n);
         else if (avg <= 39.5 && avg * 128 * 1.05 <= kGapCapNzWide) // (four threads per coordinate, ten entries each)
             e = launch_gap_stream_per<LOSS, 128, 10, kGapHotWide, kGapCapNzWide>(g, nb, lam_n);
+        else if (avg * 1.15 <= 60.0 && avg * 128 * 1.05 <= kGapCapNzWider) // (four threads per coordinate, fifteen entries each)
+            e = launch_gap_stream_per<LOSS, 128, 15, kGapHotWider, kGapCapNzWider>(g, nb, lam_n);
         else if (avg * 64 <= 3300) e = launch_gap_stream<LOSS, 64>(g, nb, lam_n);
         else if (avg * 32 <= 3300) e = launch_gap_stream<LOSS, 32>(g, nb, lam_n);
         else e = launch_gap_stream<LOSS, 16>(g, nb, lam_n);
