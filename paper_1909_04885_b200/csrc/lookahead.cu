@@ -154,6 +154,20 @@ __device__ __forceinline__ void checked_extent(const LookParams &P, int32_t &c, 
     n = (int32_t)len;
     if (!CHICLE_IN_BOUNDS(P.S.status, rs >= 0 && len >= 0 && len <= 0x7fffffff && rs + len <= P.nnz)) { rs = 0; n = 0; }
 }
+// The same search over a copy of blk_base in shared memory (a launch with at most kBaseStaged - 1 partitions; block
+// counts fit 32 bits): the dependent loads of the search cost 30 cycles each instead of an L2 round trip.
+constexpr int kBaseStaged = 260;
+__device__ __forceinline__ void block_to_part_staged(const int32_t *base, int32_t K, int64_t bid, int &k, int64_t &b)
+{
+    int32_t lo = 0, hi = K;
+    while (hi - lo > 1) {
+        const int32_t mid = (lo + hi) >> 1;
+        if ((int64_t)base[mid] <= bid) lo = mid;
+        else hi = mid;
+    }
+    k = lo;
+    b = bid - (int64_t)base[lo];
+}
 __device__ __forceinline__ void block_to_part(const LookParams &P, int64_t bid, int &k, int64_t &b)
 {
     int32_t lo = 0, hi = P.K; // blk_base[lo] <= bid < blk_base[hi] (partitions may differ in size)
@@ -281,6 +295,7 @@ template <int NZ, int HT, int THREADS> struct PreShared {
     int32_t subT[kMaxC];
     int32_t ncls[kMaxC]; // the next block's non-zeros per CTA
     int32_t total, slow, carry, ncnt;
+    int32_t base[kBaseStaged]; // blk_base of the first partitions, staged once per launch (see block_to_part_staged)
 };
 
 // One block's records (all threads of the CTA; every return below is taken by all of them).
@@ -292,7 +307,8 @@ __device__ __forceinline__ void prepare_block(const LookParams &P, const int64_t
     const int C = 1 << P.logC;
     int k;
     int64_t b;
-    block_to_part(P, bid, k, b);
+    if (P.K < kBaseStaged) block_to_part_staged(sh.base, P.K, bid, k, b);
+    else block_to_part(P, bid, k, b);
     const int64_t nk = P.S.part_off[k + 1] - P.S.part_off[k];
     const int64_t off = P.S.part_off[k] + (P.S.first_k ? P.S.first_k[k] : 0); // of this launch's first step in the order
     const int64_t steps = steps_of(P, k, nk);
@@ -785,6 +801,10 @@ __global__ void __launch_bounds__(THREADS) k_lookahead_prepare(const LookParams 
     extern __shared__ __align__(16) unsigned char smem_pre[];
     using Shared = PreShared<NZ, HT, THREADS>;
     Shared &sh = *reinterpret_cast<Shared *>(smem_pre);
+    if (P.K < kBaseStaged) {
+        for (int i = threadIdx.x; i <= P.K; i += THREADS) sh.base[i] = (int32_t)P.blk_base[i];
+        __syncthreads();
+    }
     for (int64_t bid = blockIdx.x; bid < P.n_blocks; bid += gridDim.x) {
         prepare_block<LOSS, NZ, HT, THREADS>(P, bid, sh);
         __syncthreads(); // the shared arrays are reused by the next block
