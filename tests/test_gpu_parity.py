@@ -419,6 +419,12 @@ def test_ids_beyond_the_shared_memory_part_across_slices(cluster, monkeypatch):
     run_parity(datagen.make("hinge_csr", 4 if cluster == "1" else 2), rounds=2)
 
 
+def test_more_partitions_than_the_prepare_kernel_stages_block_bases_for():
+    # up to 259 partitions the prepare kernel searches a shared-memory copy of the block bases; beyond, global memory
+    run_parity(tiny_csr(3000, 60, seed=4, K=300, density=0.1), rounds=2)
+    run_parity(tiny_csr(3000, 60, seed=4, K=259, density=0.1), rounds=2)
+
+
 def test_warp_per_coordinate_gap_kernel_on_sparse_data(monkeypatch):
     # sparse data take the streamed gap kernel by default; the warp-per-coordinate kernel stays selectable
     monkeypatch.setenv("CHICLE_FORCE_VARIANT", "gapwarp")
